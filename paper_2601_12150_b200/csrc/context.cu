@@ -1,0 +1,89 @@
+// Context, status codes and tensor-map construction (host side of libspatvit).
+#include <stdlib.h>
+#include <string.h>
+
+#include "common.cuh"
+
+extern "C" int32_t spv_create(spv_ctx** out, int32_t device) {
+  if (!out || device < 0) return SPV_ERR_INVALID_ARG;
+  *out = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || device >= n) return SPV_ERR_CUDA;
+  SPV_CUDA_OK(cudaSetDevice(device));
+  cudaDeviceProp prop;
+  SPV_CUDA_OK(cudaGetDeviceProperties(&prop, device));
+  if (prop.major != 10) return SPV_ERR_UNSUPPORTED;   // sm_100a code only
+  spv_ctx* c = (spv_ctx*)calloc(1, sizeof(spv_ctx));
+  if (!c) return SPV_ERR_CUDA;
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  if (cudaMalloc((void**)&c->d_status, 256) != cudaSuccess) { free(c); return SPV_ERR_CUDA; }
+  if (cudaMemset(c->d_status, 0, 256) != cudaSuccess) { cudaFree(c->d_status); free(c); return SPV_ERR_CUDA; }
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn) {
+    cudaFree(c->d_status);
+    free(c);
+    return SPV_ERR_CUDA;
+  }
+  c->encode_tiled = (spv_encode_tiled_fn)fn;
+  *out = c;
+  return SPV_OK;
+}
+
+extern "C" int32_t spv_destroy(spv_ctx* ctx) {
+  if (!ctx) return SPV_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaFree(ctx->d_status);
+  free(ctx);
+  return SPV_OK;
+}
+
+extern "C" const char* spv_status_string(int32_t s) {
+  switch (s) {
+    case SPV_OK: return "ok";
+    case SPV_ERR_INVALID_ARG: return "invalid argument";
+    case SPV_ERR_UNSUPPORTED: return "unsupported configuration or device";
+    case SPV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case SPV_ERR_CUDA: return "CUDA call failed";
+    case SPV_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case SPV_ERR_ALIGNMENT: return "tensor base or stride not 16-byte aligned";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int32_t spv_check(spv_ctx* ctx, void* stream) {
+  if (!ctx) return SPV_ERR_INVALID_ARG;
+  SPV_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  uint32_t st = 0;
+  SPV_CUDA_OK(cudaMemcpy(&st, ctx->d_status, sizeof(st), cudaMemcpyDeviceToHost));
+  if (st != 0) {
+    cudaMemset(ctx->d_status, 0, sizeof(st));
+    return SPV_ERR_TIMEOUT;
+  }
+  return SPV_OK;
+}
+
+extern "C" int64_t spv_launch_count(const spv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int32_t spv_make_tmap_bf16(spv_ctx* ctx, CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                           const uint64_t* strides_bytes, const uint32_t* box) {
+  if (((uintptr_t)base & 15u) != 0) return SPV_ERR_ALIGNMENT;
+  cuuint64_t gdim[5];
+  cuuint64_t gstr[4];
+  cuuint32_t bx[5], es[5];
+  for (int i = 0; i < rank; ++i) {
+    gdim[i] = dims[i];
+    bx[i] = box[i];
+    es[i] = 1;
+    if (i > 0) {
+      if (strides_bytes[i - 1] % 16 != 0) return SPV_ERR_ALIGNMENT;
+      gstr[i - 1] = strides_bytes[i - 1];
+    }
+  }
+  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, (void*)base, gdim, gstr,
+                                 bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SPV_OK : SPV_ERR_CUDA;
+}

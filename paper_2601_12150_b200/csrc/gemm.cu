@@ -1,0 +1,261 @@
+// bf16 GEMM with fused epilogues for the ViT block (QKV / out-proj / MLP / patch embedding):
+//   C[M, N] = A[M, K] * W[N, K]^T, fp32 accumulation in TMEM.
+//
+// Persistent kernel, one CTA per SM, 128 x 256 output tiles, K in slices of 64:
+//   warp 0      TMA producer (A and W slices, 128-byte swizzle, 4-stage ring)
+//   warp 1      tcgen05.mma issuer (one thread), owns the TMEM allocation (2 x 256 columns, so
+//               the epilogue of tile i overlaps the main loop of tile i+1)
+//   warps 2..5  epilogue: TMEM -> registers -> bias / activation / residual -> global
+// Rows beyond M and columns beyond N are zero-filled by TMA on load and predicated on store.
+#include "common.cuh"
+
+namespace {
+
+using namespace spv;
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_SMEM = STAGES * (A_BYTES + B_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
+
+struct EpiParams {
+  void* out;
+  int64_t ldo;
+  const float* bias;
+  const void* aux;
+  int64_t ldaux;
+  const float* scale;
+  const float* addrow;
+  int64_t ldadd;
+  int32_t rows_per_image;
+};
+
+__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+__device__ __forceinline__ float silu(float x) { return x / (1.0f + __expf(-x)); }
+
+template <int EPI>
+__device__ __forceinline__ void epilogue_store(const EpiParams& p, int m, int n0, int n_total, const uint32_t* acc) {
+  // acc: 32 fp32 accumulators of row m, columns n0 .. n0+31
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const int n = n0 + 8 * g;
+    if (n >= n_total) break;
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(acc[8 * g + i]);
+    if (p.bias) {
+      const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + n));
+      const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + n + 4));
+      v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+      v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+    }
+    if constexpr (EPI == SPV_EPI_BIAS_GELU) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = gelu_erf(v[i]);
+    } else if constexpr (EPI == SPV_EPI_BIAS_SILU) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = silu(v[i]);
+    } else if constexpr (EPI == SPV_EPI_BIAS_MUL) {
+      const uint4 a = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.aux) +
+                                                      (int64_t)m * p.ldaux + n);
+      const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&aw[i]);
+        v[2 * i] *= __low2float(h);
+        v[2 * i + 1] *= __high2float(h);
+      }
+    }
+    if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID || EPI == SPV_EPI_BIAS_ADDROW) {
+      float* o = reinterpret_cast<float*>(p.out) + (int64_t)m * p.ldo + n;
+      float4 r0, r1;
+      if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID) {
+        r0 = *reinterpret_cast<const float4*>(o);
+        r1 = *reinterpret_cast<const float4*>(o + 4);
+        float s[8] = {1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f};
+        if (p.scale) {
+          const float4 s0 = __ldg(reinterpret_cast<const float4*>(p.scale + n));
+          const float4 s1 = __ldg(reinterpret_cast<const float4*>(p.scale + n + 4));
+          s[0] = s0.x; s[1] = s0.y; s[2] = s0.z; s[3] = s0.w; s[4] = s1.x; s[5] = s1.y; s[6] = s1.z; s[7] = s1.w;
+        }
+        r0.x += s[0] * v[0]; r0.y += s[1] * v[1]; r0.z += s[2] * v[2]; r0.w += s[3] * v[3];
+        r1.x += s[4] * v[4]; r1.y += s[5] * v[5]; r1.z += s[6] * v[6]; r1.w += s[7] * v[7];
+      } else {
+        const float* ar = p.addrow + (int64_t)(m % p.rows_per_image) * p.ldadd + n;
+        const float4 a0 = __ldg(reinterpret_cast<const float4*>(ar));
+        const float4 a1 = __ldg(reinterpret_cast<const float4*>(ar + 4));
+        r0 = make_float4(v[0] + a0.x, v[1] + a0.y, v[2] + a0.z, v[3] + a0.w);
+        r1 = make_float4(v[4] + a1.x, v[5] + a1.y, v[6] + a1.z, v[7] + a1.w);
+      }
+      *reinterpret_cast<float4*>(o) = r0;
+      *reinterpret_cast<float4*>(o + 4) = r1;
+    } else {
+      uint4 w;
+      w.x = pack_bf16(v[0], v[1]);
+      w.y = pack_bf16(v[2], v[3]);
+      w.z = pack_bf16(v[4], v[5]);
+      w.w = pack_bf16(v[6], v[7]);
+      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)m * p.ldo + n) = w;
+    }
+  }
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, int M, int N,
+                 int K, EpiParams ep, uint32_t* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + STAGES * A_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_BYTES + B_BYTES));
+  uint64_t* full = bars;                 // [STAGES]  TMA -> MMA
+  uint64_t* empty = bars + STAGES;       // [STAGES]  MMA -> TMA
+  uint64_t* acc_full = bars + 2 * STAGES;       // [2] MMA -> epilogue
+  uint64_t* acc_empty = bars + 2 * STAGES + 2;  // [2] epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tiles = (M + BM - 1) / BM, n_tiles = (N + BN - 1) / BN;
+  const int tiles = m_tiles * n_tiles;
+  const int kblocks = (K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 128); }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_a);
+      tma_prefetch_desc(&tm_w);
+      uint32_t it = 0;
+      for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % STAGES;
+          mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, status, 0x100 + s);
+          mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
+          tma_load_2d(sA + s * A_BYTES, &tm_a, &full[s], kb * BK, m0);
+          tma_load_2d(sB + s * B_BYTES, &tm_w, &full[s], kb * BK, n0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16(BM, BN, false);
+      uint32_t it = 0, tcount = 0;
+      for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
+        const int a = tcount & 1;
+        mbar_wait(&acc_empty[a], ((tcount >> 1) & 1) ^ 1, abort_flag, status, 0x200 + a);
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + a * BN;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % STAGES;
+          mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, status, 0x300 + s);
+          tc_fence_after();
+          const uint64_t da = smem_desc_sw128(smem_u32(sA + s * A_BYTES));
+          const uint64_t db = smem_desc_sw128(smem_u32(sB + s * B_BYTES));
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)
+            mma_ss(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+          tc_commit(&empty[s]);
+        }
+        tc_commit(&acc_full[a]);
+      }
+    }
+  } else {
+    const int q = warp & 3;   // TMEM lane quadrant this warp may read
+    uint32_t tcount = 0;
+    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
+      const int a = tcount & 1;
+      const int m = (tile % m_tiles) * BM + q * 32 + lane;
+      const int n_base = (tile / m_tiles) * BN;
+      mbar_wait(&acc_full[a], (tcount >> 1) & 1, abort_flag, status, 0x400 + a);
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        if (n_base + c * 32 >= N) break;
+        uint32_t acc[32];
+        tmem_ld32(taddr + c * 32, acc);
+        tc_wait_ld();
+        if (m < M) epilogue_store<EPI>(ep, m, n_base + c * 32, N, acc);
+      }
+      tc_fence_before();
+      mbar_arrive(&acc_empty[a]);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+template <int EPI>
+int32_t launch(spv_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tw, const spv_gemm_desc* d, const EpiParams& ep,
+               cudaStream_t stream) {
+  static bool configured = false;
+  if (!configured) {
+    SPV_CUDA_OK(cudaFuncSetAttribute(gemm_bf16_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
+    configured = true;
+  }
+  const int tiles = ((d->m + BM - 1) / BM) * ((d->n + BN - 1) / BN);
+  const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  gemm_bf16_kernel<EPI><<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tw, d->m, d->n, d->k, ep, ctx->d_status);
+  return spv_launch_ok(ctx);
+}
+
+}  // namespace
+
+extern "C" int32_t spv_gemm_bf16(spv_ctx* ctx, const spv_gemm_desc* d, const void* a, const void* w, void* out,
+                                 void* stream_) {
+  if (!ctx || !d || !a || !w || !out) return SPV_ERR_INVALID_ARG;
+  if (d->m < 1 || d->n < 1 || d->k < 1) return SPV_ERR_INVALID_ARG;
+  if (d->k % 8 || d->n % 8 || d->lda % 8 || d->ldw % 8 || d->ldo % 8) return SPV_ERR_ALIGNMENT;
+  if (d->lda < d->k || d->ldw < d->k || d->ldo < d->n) return SPV_ERR_INVALID_ARG;
+  if (((uintptr_t)out & 15u) || ((uintptr_t)d->bias & 15u)) return SPV_ERR_ALIGNMENT;
+  EpiParams ep;
+  ep.out = out; ep.ldo = d->ldo; ep.bias = d->bias; ep.aux = d->aux; ep.ldaux = d->ldaux;
+  ep.scale = d->scale; ep.addrow = d->addrow; ep.ldadd = d->ldadd; ep.rows_per_image = d->rows_per_image;
+  if (d->epilogue == SPV_EPI_BIAS_MUL && (!d->aux || d->ldaux % 8 || ((uintptr_t)d->aux & 15u)))
+    return SPV_ERR_INVALID_ARG;
+  if (d->epilogue == SPV_EPI_BIAS_ADDROW && (!d->addrow || d->rows_per_image < 1 || d->ldadd % 4))
+    return SPV_ERR_INVALID_ARG;
+  CUtensorMap ta, tw;
+  {
+    const uint64_t dims[2] = {(uint64_t)d->k, (uint64_t)d->m};
+    const uint64_t str[1] = {(uint64_t)d->lda * 2};
+    const uint32_t box[2] = {BK, BM};
+    int32_t st = spv_make_tmap_bf16(ctx, &ta, a, 2, dims, str, box);
+    if (st != SPV_OK) return st;
+  }
+  {
+    const uint64_t dims[2] = {(uint64_t)d->k, (uint64_t)d->n};
+    const uint64_t str[1] = {(uint64_t)d->ldw * 2};
+    const uint32_t box[2] = {BK, BN};
+    int32_t st = spv_make_tmap_bf16(ctx, &tw, w, 2, dims, str, box);
+    if (st != SPV_OK) return st;
+  }
+  cudaStream_t stream = (cudaStream_t)stream_;
+  switch (d->epilogue) {
+    case SPV_EPI_BIAS: return launch<SPV_EPI_BIAS>(ctx, ta, tw, d, ep, stream);
+    case SPV_EPI_BIAS_GELU: return launch<SPV_EPI_BIAS_GELU>(ctx, ta, tw, d, ep, stream);
+    case SPV_EPI_BIAS_SILU: return launch<SPV_EPI_BIAS_SILU>(ctx, ta, tw, d, ep, stream);
+    case SPV_EPI_BIAS_MUL: return launch<SPV_EPI_BIAS_MUL>(ctx, ta, tw, d, ep, stream);
+    case SPV_EPI_BIAS_SCALE_RESID: return launch<SPV_EPI_BIAS_SCALE_RESID>(ctx, ta, tw, d, ep, stream);
+    case SPV_EPI_BIAS_ADDROW: return launch<SPV_EPI_BIAS_ADDROW>(ctx, ta, tw, d, ep, stream);
+    default: return SPV_ERR_INVALID_ARG;
+  }
+}

@@ -1,0 +1,96 @@
+// LayerNorm over fp32 residual rows, bf16 output (pre-LN of every ViT block and the final norm).
+// One warp per row, 128-bit loads, the row kept in registers between the statistics and the
+// normalisation, so each element crosses HBM once in (4 B) and once out (2 B).
+#include "common.cuh"
+
+namespace {
+
+constexpr int kMaxVec = 16;   // float4 per lane held in registers: dim <= 2048
+
+__global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict__ x, int64_t rows, int dim,
+                                                        const float* __restrict__ gamma,
+                                                        const float* __restrict__ beta, float eps,
+                                                        __nv_bfloat16* __restrict__ y,
+                                                        const int32_t* __restrict__ out_row) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  const int nvec = dim >> 2;
+  const float inv_dim = 1.0f / (float)dim;
+  for (int64_t r = warp; r < rows; r += nwarps) {
+    const float4* xr = reinterpret_cast<const float4*>(x + r * dim);
+    float4 v[kMaxVec];
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < kMaxVec; ++i) {
+      const int c = lane + 32 * i;
+      if (c < nvec) {
+        v[i] = __ldcs(xr + c);
+        sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+      }
+    }
+    for (int c = lane + 32 * kMaxVec; c < nvec; c += 32) {
+      const float4 t = xr[c];
+      sum += (t.x + t.y) + (t.z + t.w);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float mean = sum * inv_dim;
+    float sq = 0.f;
+#pragma unroll
+    for (int i = 0; i < kMaxVec; ++i) {
+      const int c = lane + 32 * i;
+      if (c < nvec) {
+        const float a = v[i].x - mean, b = v[i].y - mean, cc = v[i].z - mean, d = v[i].w - mean;
+        sq += (a * a + b * b) + (cc * cc + d * d);
+      }
+    }
+    for (int c = lane + 32 * kMaxVec; c < nvec; c += 32) {
+      const float4 t = xr[c];
+      const float a = t.x - mean, b = t.y - mean, cc = t.z - mean, d = t.w - mean;
+      sq += (a * a + b * b) + (cc * cc + d * d);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    const float rstd = rsqrtf(sq * inv_dim + eps);
+    const int64_t orow = out_row ? (int64_t)__ldg(out_row + r) : r;
+    uint2* yr = reinterpret_cast<uint2*>(y + orow * dim);
+    const float4* g4 = reinterpret_cast<const float4*>(gamma);
+    const float4* b4 = reinterpret_cast<const float4*>(beta);
+#pragma unroll
+    for (int i = 0; i < kMaxVec; ++i) {
+      const int c = lane + 32 * i;
+      if (c < nvec) {
+        const float4 g = __ldg(g4 + c), b = __ldg(b4 + c);
+        uint2 o;
+        o.x = spv::pack_bf16((v[i].x - mean) * rstd * g.x + b.x, (v[i].y - mean) * rstd * g.y + b.y);
+        o.y = spv::pack_bf16((v[i].z - mean) * rstd * g.z + b.z, (v[i].w - mean) * rstd * g.w + b.w);
+        yr[c] = o;
+      }
+    }
+    for (int c = lane + 32 * kMaxVec; c < nvec; c += 32) {
+      const float4 t = xr[c];
+      const float4 g = __ldg(g4 + c), b = __ldg(b4 + c);
+      uint2 o;
+      o.x = spv::pack_bf16((t.x - mean) * rstd * g.x + b.x, (t.y - mean) * rstd * g.y + b.y);
+      o.y = spv::pack_bf16((t.z - mean) * rstd * g.z + b.z, (t.w - mean) * rstd * g.w + b.w);
+      yr[c] = o;
+    }
+  }
+}
+
+}  // namespace
+
+extern "C" int32_t spv_layernorm(spv_ctx* ctx, const float* x, int64_t rows, int32_t dim, const float* gamma,
+                                 const float* beta, float eps, void* y, const int32_t* out_row, void* stream) {
+  if (!ctx || !x || !gamma || !beta || !y || rows < 1 || dim < 8) return SPV_ERR_INVALID_ARG;
+  if (dim % 8) return SPV_ERR_ALIGNMENT;
+  if (((uintptr_t)x & 15u) || ((uintptr_t)y & 15u) || ((uintptr_t)gamma & 15u) || ((uintptr_t)beta & 15u))
+    return SPV_ERR_ALIGNMENT;
+  int64_t blocks = (rows + 7) / 8;
+  const int64_t cap = (int64_t)ctx->sm_count * 8;
+  if (blocks > cap) blocks = cap;
+  layernorm_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(x, rows, dim, gamma, beta, eps,
+                                                                      (__nv_bfloat16*)y, out_row);
+  return spv_launch_ok(ctx);
+}
