@@ -1,4 +1,873 @@
-#include "common.cuh"
-extern "C" int32_t spv_attn_workspace_size(const spv_attn_desc*, size_t*) { return SPV_ERR_UNSUPPORTED; }
-extern "C" int32_t spatial_block_attention(spv_ctx*, const spv_attn_desc*, const void*, const void*, const void*,
-                                           void*, float*, void*, size_t, void*) { return SPV_ERR_UNSUPPORTED; }
+// Sec. 3.2 -- spatially-aware neighbouring-block sparse attention with global tokens.
+//
+// Layout idea: patch tokens are handled in BLOCK-MAJOR order (grouped by spatial block, blocks in
+// row-major order over the block grid).  The key blocks of one neighbour block row, columns
+// bx-r .. bx+r, are then ONE contiguous token range, so a key tile is a plain TMA box of
+// consecutive rows and the sparsity mask of a query row is a column interval of the tile.  The
+// same path serves full grids, ragged edge blocks and filtered token sets (blocks that lost
+// tokens just have shorter ranges).  Neighbour ranges are computed on the fly from block
+// coordinates and the per-block offsets; no N x N object and no neighbour list exists.
+//
+// Kernels
+//   attn_plan_*        per-block token counts (binary search in the sorted positions), scan,
+//                      greedy packing of consecutive blocks into <=128-row query tiles
+//   attn_regroup       row-major -> block-major copy of Q, K, V (only for row-major callers)
+//   attn_patch_kernel  flash-style tcgen05 kernel: S = Q K^T into TMEM, online softmax by 128
+//                      row-owning threads, P written back to TMEM as bf16, O += P V with V as an
+//                      MN-major shared-memory operand; global tokens enter as the initial
+//                      softmax state, so key tiles stay multiples of the MMA shape
+//   attn_global_*      the dense rows of the global (CLS) queries and the CLS->patch scores
+#include "attention.cuh"
+
+namespace {
+
+using namespace spv;
+
+constexpr int TQ = 128;            // query rows per tile (MMA M)
+constexpr int TK = 128;            // keys per tile (MMA N of S, K extent of P V)
+constexpr int HD = 64;             // head_dim
+constexpr int KST = 2;             // K / V smem stages
+constexpr int ATT_THREADS = 192;   // warps 0-3 softmax, 4 TMA, 5 MMA
+constexpr int TILE_BYTES = 128 * 128;
+constexpr int ATT_SMEM = TILE_BYTES * (1 + 2 * KST) + 1024 + 256;
+constexpr int MAXG = 8;
+constexpr uint32_t TMEM_COLS = 256;
+constexpr uint32_t S_COL = 0, P_COL = 128, O_COL = 192;
+
+// ------------------------------------------------------------------------------------------
+// plan
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int lower_bound_i32(const int32_t* a, int n, int key) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (__ldg(a + mid) < key) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ int block_of_pos(int pos, int W, int b, int nbx) {
+  return ((pos / W) / b) * nbx + (pos % W) / b;
+}
+
+// first ordinal t whose block id is >= blk (token order block-major, so block ids are sorted)
+__device__ __forceinline__ int lower_bound_blk(const int32_t* pos, int n, int blk, int W, int b, int nbx) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (block_of_pos(__ldg(pos + mid), W, b, nbx) < blk) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+// One thread per search segment.  Row-major callers: segment = (block, row inside block): its
+// tokens are one run of the position-sorted input.  Block-major callers: segment = block.
+__global__ void attn_plan_segments(SpvAttnPlan p, const int32_t* __restrict__ patch_pos, int token_order) {
+  const int seg = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = blockIdx.y;
+  if (seg >= p.nseg) return;
+  const int blk = seg / p.segs_per_block, yy = seg % p.segs_per_block;
+  const int by = blk / p.nbx, bx = blk % p.nbx;
+  const int32_t* pos = patch_pos ? patch_pos + (size_t)b * p.n_patch : nullptr;
+  int lo, cnt;
+  if (token_order == SPV_TOKENS_ROW_MAJOR) {
+    const int y = by * p.block + yy;
+    const int x0 = bx * p.block, x1 = min(x0 + p.block, p.grid_w);
+    if (y >= p.grid_h) { lo = 0; cnt = 0; }
+    else if (pos) {
+      lo = lower_bound_i32(pos, p.n_patch, y * p.grid_w + x0);
+      cnt = lower_bound_i32(pos, p.n_patch, y * p.grid_w + x1) - lo;
+    } else { lo = y * p.grid_w + x0; cnt = x1 - x0; }
+  } else {
+    if (pos) {
+      lo = lower_bound_blk(pos, p.n_patch, blk, p.grid_w, p.block, p.nbx);
+      cnt = lower_bound_blk(pos, p.n_patch, blk + 1, p.grid_w, p.block, p.nbx) - lo;
+    } else {   // full grid already grouped by block: sizes follow from the geometry
+      const int bh = min(p.block, p.grid_h - by * p.block), bw = min(p.block, p.grid_w - bx * p.block);
+      cnt = bh * bw;
+      lo = 0;   // filled by the scan (identity)
+    }
+  }
+  p.seg_lo[(size_t)b * p.nseg + seg] = lo;
+  p.seg_cnt[(size_t)b * p.nseg + seg] = cnt;
+}
+
+// One CTA per image: exclusive scan of the segment counts, block offsets, then the query tiles:
+// per block row, consecutive blocks are packed greedily into tiles of at most TQ tokens; a block
+// larger than TQ is cut into TQ-row pieces.
+__global__ void __launch_bounds__(1024) attn_plan_scan(SpvAttnPlan p) {
+  __shared__ int warp_sums[32];
+  __shared__ int carry;
+  const int b = blockIdx.x;
+  const int32_t* cnt = p.seg_cnt + (size_t)b * p.nseg;
+  int32_t* off = p.seg_off + (size_t)b * (p.nseg + 1);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < p.nseg; base += 1024) {
+    const int i = base + threadIdx.x;
+    const int v = i < p.nseg ? cnt[i] : 0;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { int n = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += n; }
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      int w = warp_sums[lane], s = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { int n = __shfl_up_sync(0xffffffffu, s, o); if (lane >= o) s += n; }
+      warp_sums[lane] = s - w;
+    }
+    __syncthreads();
+    const int excl = carry + warp_sums[warp] + inc - v;
+    if (i < p.nseg) off[i] = excl;
+    __syncthreads();
+    if (threadIdx.x == 1023) carry = excl + v;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) off[p.nseg] = carry;
+  __syncthreads();
+  int32_t* boff = p.block_off + (size_t)b * (p.nb + 1);
+  for (int blk = threadIdx.x; blk <= p.nb; blk += 1024) boff[blk] = off[min(blk * p.segs_per_block, p.nseg)];
+  __syncthreads();
+  int4* tiles = p.tiles + (size_t)b * p.tiles_per_image;
+  for (int by = threadIdx.x; by < p.nby; by += 1024) {
+    int4* t = tiles + (size_t)by * p.tiles_per_row;
+    int nt = 0;
+    int cur_begin = -1, cur_end = 0, cur_first = 0, cur_last = 0;
+    for (int bx = 0; bx < p.nbx; ++bx) {
+      int s = boff[by * p.nbx + bx];
+      const int e = boff[by * p.nbx + bx + 1];
+      if (e == s) continue;
+      if (cur_begin >= 0 && (e - cur_begin) <= TQ) { cur_end = e; cur_last = bx; continue; }
+      if (cur_begin >= 0) { t[nt++] = make_int4(cur_begin, cur_end, by, cur_first | (cur_last << 16)); cur_begin = -1; }
+      while (e - s > TQ) { t[nt++] = make_int4(s, s + TQ, by, bx | (bx << 16)); s += TQ; }
+      cur_begin = s; cur_end = e; cur_first = bx; cur_last = bx;
+    }
+    if (cur_begin >= 0) t[nt++] = make_int4(cur_begin, cur_end, by, cur_first | (cur_last << 16));
+    for (; nt < p.tiles_per_row; ++nt) t[nt] = make_int4(0, 0, 0, 0);
+  }
+}
+
+__global__ void attn_plan_fill(SpvAttnPlan p) {
+  const int seg = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = blockIdx.y;
+  if (seg >= p.nseg) return;
+  const int off = p.seg_off[(size_t)b * (p.nseg + 1) + seg];
+  const int cnt = p.seg_cnt[(size_t)b * p.nseg + seg];
+  const int lo = p.seg_lo[(size_t)b * p.nseg + seg];
+  const int blk = seg / p.segs_per_block;
+  for (int e = 0; e < cnt; ++e) {
+    p.tok_blk[(size_t)b * p.n_patch + off + e] = blk;
+    if (!p.identity) p.bm_src[(size_t)b * p.n_patch + off + e] = lo + e;
+  }
+}
+
+// Q, K, V rows of every (token, head) copied into block-major order: 8 lanes move one 128-byte row.
+__global__ void __launch_bounds__(256) attn_regroup(const __nv_bfloat16* __restrict__ q,
+                                                    const __nv_bfloat16* __restrict__ k,
+                                                    const __nv_bfloat16* __restrict__ v, int64_t sb, int64_t st,
+                                                    int64_t sh, __nv_bfloat16* __restrict__ qo,
+                                                    __nv_bfloat16* __restrict__ ko, __nv_bfloat16* __restrict__ vo,
+                                                    const int32_t* __restrict__ bm_src, int batch, int n_global,
+                                                    int n_patch, int heads) {
+  const int n_tok = n_global + n_patch;
+  const int64_t total = (int64_t)batch * n_tok * heads;
+  const int sub = threadIdx.x & 7;
+  for (int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 3; r < total;
+       r += ((int64_t)gridDim.x * blockDim.x) >> 3) {
+    const int h = (int)(r % heads);
+    const int64_t bt = r / heads;
+    const int t = (int)(bt % n_tok), b = (int)(bt / n_tok);
+    const int src = t < n_global ? t : n_global + __ldg(bm_src + (size_t)b * n_patch + (t - n_global));
+    const int64_t so = b * sb + (int64_t)src * st + (int64_t)h * sh + sub * 8;
+    const int64_t dof = (((int64_t)b * n_tok + t) * heads + h) * HD + sub * 8;
+    *reinterpret_cast<uint4*>(qo + dof) = __ldg(reinterpret_cast<const uint4*>(q + so));
+    *reinterpret_cast<uint4*>(ko + dof) = __ldg(reinterpret_cast<const uint4*>(k + so));
+    *reinterpret_cast<uint4*>(vo + dof) = __ldg(reinterpret_cast<const uint4*>(v + so));
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// patch-query kernel
+// ------------------------------------------------------------------------------------------
+struct PatchParams {
+  const int32_t* block_off;
+  const int32_t* tok_blk;
+  const int4* tiles;
+  const int32_t* o_tok;
+  const __nv_bfloat16 *k, *v;
+  int64_t sb, st, sh;
+  __nv_bfloat16* o;
+  int64_t o_sb, o_st, o_sh;
+  int nbx, nby, nb, radius, n_global, n_patch, tiles_per_image;
+  float scale_log2;
+  uint32_t* status;
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ void unpack8(const uint4& u, float* f) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&w[i]);
+    f[2 * i] = __low2float(h);
+    f[2 * i + 1] = __high2float(h);
+  }
+}
+
+__global__ void __launch_bounds__(ATT_THREADS, 2)
+attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                  const __grid_constant__ CUtensorMap tm_v, const PatchParams p) {
+  const int b = blockIdx.z, h = blockIdx.y;
+  const int4 tile = __ldg(p.tiles + (size_t)b * p.tiles_per_image + blockIdx.x);
+  const int q_begin = tile.x, q_end = tile.y;
+  if (q_begin >= q_end) return;                          // unused slot of the tile table
+  const int by = tile.z, bx_first = tile.w & 0xFFFF, bx_last = tile.w >> 16;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;
+  uint8_t* sK = smem + TILE_BYTES;
+  uint8_t* sV = smem + TILE_BYTES * (1 + KST);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + TILE_BYTES * (1 + 2 * KST));
+  uint64_t* q_full = bars;
+  uint64_t* k_full = bars + 1;
+  uint64_t* k_empty = k_full + KST;
+  uint64_t* v_full = k_empty + KST;
+  uint64_t* v_empty = v_full + KST;
+  uint64_t* s_full = v_empty + KST;
+  uint64_t* s_free = s_full + 1;
+  uint64_t* p_full = s_free + 1;
+  uint64_t* pv_done = p_full + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + 1);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = p.radius, G = p.n_global;
+  const int cy0 = max(by - r, 0), cy1 = min(by + r, p.nby - 1);
+  const int cxl = max(bx_first - r, 0), cxh = min(bx_last + r, p.nbx - 1);
+  const int32_t* boff = p.block_off + (size_t)b * (p.nb + 1);
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int s = 0; s < KST; ++s) {
+      mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
+      mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
+    }
+    mbar_init(s_full, 1);
+    mbar_init(s_free, 128);
+    mbar_init(p_full, 128);
+    mbar_init(pv_done, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 5) {
+    tmem_alloc(tmem_slot, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 4) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
+      mbar_expect_tx(q_full, TILE_BYTES);
+      tma_load_4d(sQ, &tm_q, q_full, 0, G + q_begin, h, b);
+      uint32_t j = 0;
+      for (int cy = cy0; cy <= cy1; ++cy) {
+        const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
+        for (int kb = ks; kb < ke; kb += TK, ++j) {
+          const int s = j % KST;
+          const uint32_t ph = ((j / KST) & 1) ^ 1;
+          mbar_wait(&k_empty[s], ph, abort_flag, p.status, 0x1100 + s);
+          mbar_expect_tx(&k_full[s], TILE_BYTES);
+          tma_load_4d(sK + s * TILE_BYTES, &tm_k, &k_full[s], 0, G + kb, h, b);
+          mbar_wait(&v_empty[s], ph, abort_flag, p.status, 0x1200 + s);
+          mbar_expect_tx(&v_full[s], TILE_BYTES);
+          tma_load_4d(sV + s * TILE_BYTES, &tm_v, &v_full[s], 0, G + kb, h, b);
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      uint32_t n_kv = 0;
+      for (int cy = cy0; cy <= cy1; ++cy) {
+        const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
+        n_kv += (uint32_t)((ke - ks + TK - 1) / TK);
+      }
+      constexpr uint32_t idesc_s = idesc_bf16(TQ, TK, false);
+      constexpr uint32_t idesc_o = idesc_bf16(TQ, HD, true);
+      const uint64_t dq = smem_desc_sw128(smem_u32(sQ));
+      auto issue_qk = [&](uint32_t j) {
+        const int s = j % KST;
+        mbar_wait(&k_full[s], (j / KST) & 1, abort_flag, p.status, 0x1300 + s);
+        if (j > 0) mbar_wait(s_free, (j - 1) & 1, abort_flag, p.status, 0x1400);
+        tc_fence_after();
+        const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * TILE_BYTES));
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk)
+          mma_ss(tmem + S_COL, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_s, kk != 0);
+        tc_commit(s_full);
+        tc_commit(&k_empty[s]);
+      };
+      mbar_wait(q_full, 0, abort_flag, p.status, 0x1000);
+      if (n_kv > 0) issue_qk(0);
+      for (uint32_t j = 0; j < n_kv; ++j) {
+        if (j + 1 < n_kv) issue_qk(j + 1);
+        const int s = j % KST;
+        mbar_wait(&v_full[s], (j / KST) & 1, abort_flag, p.status, 0x1500 + s);
+        mbar_wait(p_full, j & 1, abort_flag, p.status, 0x1600);
+        tc_fence_after();
+        const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * TILE_BYTES));
+#pragma unroll
+        for (int kk = 0; kk < TK / 16; ++kk)
+          mma_ts(tmem + O_COL, tmem + P_COL + kk * 8, dv + (uint64_t)(kk * 128), idesc_o, (j | kk) != 0);
+        tc_commit(pv_done);
+        tc_commit(&v_empty[s]);
+      }
+    }
+  } else {
+    // ---------------- softmax + epilogue: thread `row` owns query row `row` (TMEM lane `row`)
+    const int row = threadIdx.x;
+    const int tok = q_begin + row;
+    const bool valid = tok < q_end;
+    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    int bxq = bx_first;
+    if (valid) bxq = __ldg(p.tok_blk + (size_t)b * p.n_patch + tok) % p.nbx;
+    const int rlo = max(bxq - r, 0), rhi = min(bxq + r, p.nbx - 1);
+    const float sl2 = p.scale_log2;
+
+    // global tokens: initial softmax state (m, l); their value rows are added in the epilogue
+    mbar_wait(q_full, 0, abort_flag, p.status, 0x1700);
+    float sg[MAXG];
+    float m = -INFINITY;
+    {
+      float qf[HD];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 u = *reinterpret_cast<const uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4));
+        unpack8(u, qf + 8 * c);
+      }
+#pragma unroll
+      for (int g = 0; g < MAXG; ++g) {
+        sg[g] = -INFINITY;
+        if (g < G) {
+          const uint4* kg = reinterpret_cast<const uint4*>(p.k + b * p.sb + (int64_t)g * p.st + (int64_t)h * p.sh);
+          float dot = 0.f;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            float kf[8];
+            unpack8(__ldg(kg + c), kf);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dot = fmaf(qf[8 * c + i], kf[i], dot);
+          }
+          sg[g] = dot * sl2;
+          m = fmaxf(m, sg[g]);
+        }
+      }
+    }
+    float l = 0.f;
+#pragma unroll
+    for (int g = 0; g < MAXG; ++g) if (g < G) l += fast_exp2(sg[g] - m);
+
+    uint32_t j = 0;
+    for (int cy = cy0; cy <= cy1; ++cy) {
+      const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
+      int lo = __ldg(boff + cy * p.nbx + rlo), hi = __ldg(boff + cy * p.nbx + rhi + 1);
+      if (!valid) hi = lo;
+      for (int kb = ks; kb < ke; kb += TK, ++j) {
+        // this row's allowed keys are the tile columns [c_lo, c_hi)
+        const int c_lo = min(max(lo - kb, 0), TK), c_hi = min(max(hi - kb, 0), TK);
+        const bool some = c_lo < c_hi;
+        int w_lo = some ? c_lo : TK, w_hi = some ? c_hi : 0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          w_lo = min(w_lo, __shfl_xor_sync(0xffffffffu, w_lo, o));
+          w_hi = max(w_hi, __shfl_xor_sync(0xffffffffu, w_hi, o));
+        }
+        mbar_wait(s_full, j & 1, abort_flag, p.status, 0x1800);
+        tc_fence_after();
+        // pass 1: row maximum over the allowed columns
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < TK / 32; ++c) {
+          if (32 * c < w_hi && 32 * c + 32 > w_lo) {
+            uint32_t sr[32];
+            tmem_ld32(lane_addr + S_COL + 32 * c, sr);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int col = 32 * c + i;
+              if (col >= c_lo && col < c_hi) mx = fmaxf(mx, __uint_as_float(sr[i]));
+            }
+          }
+        }
+        // lazy rescale: the running maximum only moves when it would grow by more than 2^8
+        const float m_t = mx * sl2;
+        const bool need = m_t > m + 8.0f;
+        const float m_new = need ? m_t : m;
+        const float alpha = need ? fast_exp2(m - m_new) : 1.0f;
+        const bool any_need = __any_sync(0xffffffffu, need);
+        // pass 2: p = 2^(s*scale - m), packed to bf16 pairs
+        uint32_t pk[TK / 2];
+        float rowsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < TK / 32; ++c) {
+          if (32 * c < w_hi && 32 * c + 32 > w_lo) {
+            uint32_t sr[32];
+            tmem_ld32(lane_addr + S_COL + 32 * c, sr);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              const int col = 32 * c + i;
+              float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), sl2, -m_new));
+              float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), sl2, -m_new));
+              if (!(col >= c_lo && col < c_hi)) p0 = 0.f;
+              if (!(col + 1 >= c_lo && col + 1 < c_hi)) p1 = 0.f;
+              rowsum += p0 + p1;
+              pk[16 * c + i / 2] = pack_bf16(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[16 * c + i] = 0u;
+          }
+        }
+        l = l * alpha + rowsum;
+        m = m_new;
+        tc_fence_before();
+        mbar_arrive(s_free);                               // S may be overwritten by the next Q K^T
+        if (j > 0) {
+          mbar_wait(pv_done, (j - 1) & 1, abort_flag, p.status, 0x1900);   // P buffer and O are free
+          tc_fence_after();
+          if (any_need) {
+#pragma unroll
+            for (int c = 0; c < HD / 32; ++c) {
+              uint32_t orr[32];
+              tmem_ld32(lane_addr + O_COL + 32 * c, orr);
+              tc_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+              tmem_st32(lane_addr + O_COL + 32 * c, orr);
+            }
+          }
+        }
+#pragma unroll
+        for (int c = 0; c < TK / 32; ++c) tmem_st16(lane_addr + P_COL + 16 * c, pk + 16 * c);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(p_full);
+      }
+    }
+    // ---------------- epilogue: O / l with the global tokens' share added
+    if (j > 0) {
+      mbar_wait(pv_done, (j - 1) & 1, abort_flag, p.status, 0x1A00);
+      tc_fence_after();
+    }
+    float of[HD];
+#pragma unroll
+    for (int c = 0; c < HD / 32; ++c) {
+      uint32_t orr[32];
+      if (j > 0) {
+        tmem_ld32(lane_addr + O_COL + 32 * c, orr);
+        tc_wait_ld();
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) orr[i] = 0u;
+      }
+#pragma unroll
+      for (int i = 0; i < 32; ++i) of[32 * c + i] = __uint_as_float(orr[i]);
+    }
+#pragma unroll
+    for (int g = 0; g < MAXG; ++g) {
+      if (g < G) {
+        const float w = fast_exp2(sg[g] - m);
+        const uint4* vg = reinterpret_cast<const uint4*>(p.v + b * p.sb + (int64_t)g * p.st + (int64_t)h * p.sh);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          float vf[8];
+          unpack8(__ldg(vg + c), vf);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) of[8 * c + i] = fmaf(w, vf[i], of[8 * c + i]);
+        }
+      }
+    }
+    if (valid) {
+      const float inv = 1.0f / l;
+      const int ot = p.o_tok ? __ldg(p.o_tok + (size_t)b * p.n_patch + tok) : tok;
+      uint4* dst = reinterpret_cast<uint4*>(p.o + b * p.o_sb + (int64_t)(G + ot) * p.o_st + (int64_t)h * p.o_sh);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint4 w;
+        w.x = pack_bf16(of[8 * c] * inv, of[8 * c + 1] * inv);
+        w.y = pack_bf16(of[8 * c + 2] * inv, of[8 * c + 3] * inv);
+        w.z = pack_bf16(of[8 * c + 4] * inv, of[8 * c + 5] * inv);
+        w.w = pack_bf16(of[8 * c + 6] * inv, of[8 * c + 7] * inv);
+        dst[c] = w;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 5) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+// ------------------------------------------------------------------------------------------
+// global-query rows
+// ------------------------------------------------------------------------------------------
+constexpr int GCH = 512;   // keys per CTA
+
+// grid (chunks, heads, batch * G).  Writes scaled logits, and per chunk (max, sum, sum p*v).
+__global__ void __launch_bounds__(256) attn_global_partial(const __nv_bfloat16* __restrict__ q,
+                                                           const __nv_bfloat16* __restrict__ k,
+                                                           const __nv_bfloat16* __restrict__ v, int64_t sb,
+                                                           int64_t st, int64_t sh, int n_tok, int n_global,
+                                                           int heads, float scale, float* __restrict__ logits,
+                                                           float* __restrict__ part_ml, float* __restrict__ part_o,
+                                                           int n_chunks) {
+  __shared__ float s_s[GCH];
+  __shared__ float s_red[32];
+  __shared__ float s_o[32][HD + 1];
+  const int chunk = blockIdx.x, h = blockIdx.y, bg = blockIdx.z;
+  const int b = bg / n_global, g = bg % n_global;
+  const int k0 = chunk * GCH, k1 = min(k0 + GCH, n_tok);
+  const int sub = threadIdx.x & 7, grp = threadIdx.x >> 3;   // 8 lanes per key, 32 keys in flight
+  float qf[8];
+  unpack8(__ldg(reinterpret_cast<const uint4*>(q + b * sb + (int64_t)g * st + (int64_t)h * sh) + sub), qf);
+  for (int i = threadIdx.x; i < GCH; i += 256) s_s[i] = -INFINITY;
+  __syncthreads();
+  float lmax = -INFINITY;
+  for (int kk = k0 + grp; kk < k1; kk += 32) {
+    float kf[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(k + b * sb + (int64_t)kk * st + (int64_t)h * sh) + sub), kf);
+    float d = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) d = fmaf(qf[i], kf[i], d);
+    d += __shfl_xor_sync(0xffffffffu, d, 1);
+    d += __shfl_xor_sync(0xffffffffu, d, 2);
+    d += __shfl_xor_sync(0xffffffffu, d, 4);
+    d *= scale;
+    if (sub == 0) s_s[kk - k0] = d;
+    lmax = fmaxf(lmax, d);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) lmax = fmaxf(lmax, __shfl_xor_sync(0xffffffffu, lmax, o));
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = lmax;
+  __syncthreads();
+  float cmax = s_red[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) cmax = fmaxf(cmax, s_red[w]);
+  float* lg = logits + ((size_t)bg * heads + h) * n_tok;
+  float lsum = 0.f;
+  for (int i = threadIdx.x; i < k1 - k0; i += 256) {
+    const float s = s_s[i];
+    lg[k0 + i] = s;
+    lsum += __expf(s - cmax);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) s_red[8 + (threadIdx.x >> 5)] = lsum;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int kk = k0 + grp; kk < k1; kk += 32) {
+    const float pw = __expf(s_s[kk - k0] - cmax);
+    float vf[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(v + b * sb + (int64_t)kk * st + (int64_t)h * sh) + sub), vf);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = fmaf(pw, vf[i], acc[i]);
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) s_o[grp][sub * 8 + i] = acc[i];
+  __syncthreads();
+  const size_t pidx = ((size_t)bg * heads + h) * n_chunks + chunk;
+  if (threadIdx.x < HD) {
+    float t = 0.f;
+#pragma unroll
+    for (int gI = 0; gI < 32; ++gI) t += s_o[gI][threadIdx.x];
+    part_o[pidx * HD + threadIdx.x] = t;
+  }
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) t += s_red[8 + w];
+    part_ml[pidx * 2] = cmax;
+    part_ml[pidx * 2 + 1] = t;
+  }
+}
+
+// grid (heads, batch * G): merge the chunk partials, write the output row and (g == 0) the
+// CLS->patch softmax weights.
+__global__ void __launch_bounds__(256) attn_global_combine(const float* __restrict__ logits,
+                                                           const float* __restrict__ part_ml,
+                                                           const float* __restrict__ part_o, int n_chunks,
+                                                           int n_tok, int n_global, int heads,
+                                                           __nv_bfloat16* __restrict__ o, int64_t o_sb,
+                                                           int64_t o_st, int64_t o_sh, float* __restrict__ scores,
+                                                           const int32_t* __restrict__ score_idx) {
+  __shared__ float s_m, s_l;
+  __shared__ float s_red[16];
+  const int h = blockIdx.x, bg = blockIdx.y;
+  const int b = bg / n_global, g = bg % n_global;
+  const size_t pbase = ((size_t)bg * heads + h) * n_chunks;
+  float mx = -INFINITY;
+  for (int c = threadIdx.x; c < n_chunks; c += 256) mx = fmaxf(mx, part_ml[(pbase + c) * 2]);
+#pragma unroll
+  for (int o2 = 16; o2 > 0; o2 >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o2));
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = s_red[0];
+    for (int w = 1; w < 8; ++w) t = fmaxf(t, s_red[w]);
+    s_m = t;
+  }
+  __syncthreads();
+  const float M = s_m;
+  float ls = 0.f;
+  for (int c = threadIdx.x; c < n_chunks; c += 256)
+    ls += part_ml[(pbase + c) * 2 + 1] * __expf(part_ml[(pbase + c) * 2] - M);
+#pragma unroll
+  for (int o2 = 16; o2 > 0; o2 >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o2);
+  if ((threadIdx.x & 31) == 0) s_red[8 + (threadIdx.x >> 5)] = ls;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < 8; ++w) t += s_red[8 + w];
+    s_l = t;
+  }
+  __syncthreads();
+  const float inv = 1.0f / s_l;
+  if (threadIdx.x < HD) {
+    float acc = 0.f;
+    for (int c = 0; c < n_chunks; ++c)
+      acc += part_o[(pbase + c) * HD + threadIdx.x] * __expf(part_ml[(pbase + c) * 2] - M);
+    o[b * o_sb + (int64_t)g * o_st + (int64_t)h * o_sh + threadIdx.x] = __float2bfloat16(acc * inv);
+  }
+  if (scores && g == 0) {
+    const float* lg = logits + ((size_t)bg * heads + h) * n_tok;
+    const int n_patch = n_tok - n_global;
+    float* sc = scores + ((size_t)b * heads + h) * n_patch;
+    for (int t = threadIdx.x; t < n_patch; t += 256) {
+      const int dst = score_idx ? __ldg(score_idx + (size_t)b * n_patch + t) : t;
+      sc[dst] = __expf(lg[n_global + t] - M) * inv;
+    }
+  }
+}
+
+int32_t make_qkv_map(spv_ctx* ctx, CUtensorMap* m, const void* base, int64_t sb, int64_t st, int64_t sh, int n_tok,
+                     int heads, int batch, int rows) {
+  const uint64_t dims[4] = {(uint64_t)HD, (uint64_t)n_tok, (uint64_t)heads, (uint64_t)batch};
+  const uint64_t str[3] = {(uint64_t)st * 2, (uint64_t)sh * 2, (uint64_t)sb * 2};
+  const uint32_t box[4] = {(uint32_t)HD, (uint32_t)rows, 1, 1};
+  return spv_make_tmap_bf16(ctx, m, base, 4, dims, str, box);
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+static void plan_geometry(SpvAttnPlan* p, int token_order) {
+  p->nby = (p->grid_h + p->block - 1) / p->block;
+  p->nbx = (p->grid_w + p->block - 1) / p->block;
+  p->nb = p->nby * p->nbx;
+  p->segs_per_block = token_order == SPV_TOKENS_ROW_MAJOR ? p->block : 1;
+  p->nseg = p->nb * p->segs_per_block;
+  const int64_t rowcap = (int64_t)(p->block < p->grid_h ? p->block : p->grid_h) * p->grid_w;
+  const int64_t full = (rowcap + TQ - 1) / TQ;
+  int64_t t = 2 * full + 1;
+  if (p->nbx + full < t) t = p->nbx + full;
+  p->tiles_per_row = (int32_t)t;
+  p->tiles_per_image = p->tiles_per_row * p->nby;
+  p->identity = token_order == SPV_TOKENS_BLOCK_MAJOR;
+}
+
+size_t spv_attn_plan_bytes(int32_t batch, int32_t grid_h, int32_t grid_w, int32_t block, int32_t n_patch,
+                           int32_t token_order) {
+  SpvAttnPlan p{};
+  p.batch = batch; p.grid_h = grid_h; p.grid_w = grid_w; p.block = block; p.n_patch = n_patch;
+  plan_geometry(&p, token_order);
+  size_t n = 0;
+  n += spv_align_up((size_t)batch * p.nseg * 4, 256) * 2;
+  n += spv_align_up((size_t)batch * (p.nseg + 1) * 4, 256);
+  n += spv_align_up((size_t)batch * (p.nb + 1) * 4, 256);
+  n += spv_align_up((size_t)batch * n_patch * 4, 256) * 2;
+  n += spv_align_up((size_t)batch * p.tiles_per_image * sizeof(int4), 256);
+  return n;
+}
+
+int32_t spv_attn_plan_build(spv_ctx* ctx, int32_t batch, int32_t grid_h, int32_t grid_w, int32_t block,
+                            int32_t radius, int32_t n_global, int32_t n_patch, const int32_t* patch_pos,
+                            int32_t token_order, void* ws, size_t ws_bytes, cudaStream_t stream,
+                            SpvAttnPlan* plan) {
+  SpvAttnPlan p{};
+  p.batch = batch; p.grid_h = grid_h; p.grid_w = grid_w; p.block = block; p.n_global = n_global;
+  p.n_patch = n_patch;
+  plan_geometry(&p, token_order);
+  const int reach = (p.nby > p.nbx ? p.nby : p.nbx);
+  p.radius = radius < reach ? radius : reach;
+  if (p.nbx >= 65536) return SPV_ERR_UNSUPPORTED;
+  if (ws_bytes < spv_attn_plan_bytes(batch, grid_h, grid_w, block, n_patch, token_order)) return SPV_ERR_WORKSPACE;
+  char* w = (char*)ws;
+  auto take = [&](size_t bytes) { void* r = w; w += spv_align_up(bytes, 256); return r; };
+  p.seg_lo = (int32_t*)take((size_t)batch * p.nseg * 4);
+  p.seg_cnt = (int32_t*)take((size_t)batch * p.nseg * 4);
+  p.seg_off = (int32_t*)take((size_t)batch * (p.nseg + 1) * 4);
+  p.block_off = (int32_t*)take((size_t)batch * (p.nb + 1) * 4);
+  p.tok_blk = (int32_t*)take((size_t)batch * n_patch * 4);
+  p.bm_src = (int32_t*)take((size_t)batch * n_patch * 4);
+  p.tiles = (int4*)take((size_t)batch * p.tiles_per_image * sizeof(int4));
+  const dim3 sgrid((p.nseg + 255) / 256, batch);
+  attn_plan_segments<<<sgrid, 256, 0, stream>>>(p, patch_pos, token_order);
+  attn_plan_scan<<<batch, 1024, 0, stream>>>(p);
+  attn_plan_fill<<<sgrid, 256, 0, stream>>>(p);
+  *plan = p;
+  return spv_launch_ok(ctx, 3);
+}
+
+int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, cudaStream_t stream) {
+  static bool configured = false;
+  if (!configured) {
+    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM));
+    configured = true;
+  }
+  const int n_tok = plan->n_global + plan->n_patch;
+  CUtensorMap tq, tk, tv;
+  int32_t st;
+  if ((st = make_qkv_map(ctx, &tq, io->q, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TQ)) != SPV_OK) return st;
+  if ((st = make_qkv_map(ctx, &tk, io->k, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TK)) != SPV_OK) return st;
+  if ((st = make_qkv_map(ctx, &tv, io->v, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TK)) != SPV_OK) return st;
+  PatchParams pp;
+  pp.block_off = plan->block_off; pp.tok_blk = plan->tok_blk; pp.tiles = plan->tiles; pp.o_tok = io->o_tok;
+  pp.k = (const __nv_bfloat16*)io->k; pp.v = (const __nv_bfloat16*)io->v;
+  pp.sb = io->sb; pp.st = io->st; pp.sh = io->sh;
+  pp.o = (__nv_bfloat16*)io->o; pp.o_sb = io->o_sb; pp.o_st = io->o_st; pp.o_sh = io->o_sh;
+  pp.nbx = plan->nbx; pp.nby = plan->nby; pp.nb = plan->nb; pp.radius = plan->radius;
+  pp.n_global = plan->n_global; pp.n_patch = plan->n_patch; pp.tiles_per_image = plan->tiles_per_image;
+  pp.scale_log2 = io->scale * 1.4426950408889634f;
+  pp.status = ctx->d_status;
+  const dim3 grid(plan->tiles_per_image, io->heads, plan->batch);
+  attn_patch_kernel<<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, pp);
+  return spv_launch_ok(ctx);
+}
+
+size_t spv_attn_global_bytes(int32_t batch, int32_t n_global, int32_t heads, int32_t n_tok) {
+  const size_t rows = (size_t)batch * n_global * heads;
+  const size_t chunks = (n_tok + GCH - 1) / GCH;
+  return spv_align_up(rows * n_tok * 4, 256) + spv_align_up(rows * chunks * 2 * 4, 256) +
+         spv_align_up(rows * chunks * HD * 4, 256);
+}
+
+int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, float* scores,
+                             const int32_t* score_idx, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  const int n_tok = plan->n_global + plan->n_patch, G = plan->n_global, B = plan->batch;
+  if (ws_bytes < spv_attn_global_bytes(B, G, io->heads, n_tok)) return SPV_ERR_WORKSPACE;
+  const size_t rows = (size_t)B * G * io->heads;
+  const int chunks = (n_tok + GCH - 1) / GCH;
+  char* w = (char*)ws;
+  float* logits = (float*)w; w += spv_align_up(rows * n_tok * 4, 256);
+  float* part_ml = (float*)w; w += spv_align_up(rows * chunks * 2 * 4, 256);
+  float* part_o = (float*)w;
+  attn_global_partial<<<dim3(chunks, io->heads, B * G), 256, 0, stream>>>(
+      (const __nv_bfloat16*)io->q, (const __nv_bfloat16*)io->k, (const __nv_bfloat16*)io->v, io->sb, io->st, io->sh,
+      n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks);
+  attn_global_combine<<<dim3(io->heads, B * G), 256, 0, stream>>>(logits, part_ml, part_o, chunks, n_tok, G,
+                                                                 io->heads, (__nv_bfloat16*)io->o, io->o_sb,
+                                                                 io->o_st, io->o_sh, scores, score_idx);
+  return spv_launch_ok(ctx, 2);
+}
+
+// ------------------------------------------------------------------------------------------
+// C entry points
+// ------------------------------------------------------------------------------------------
+static int32_t validate_desc(const spv_attn_desc* d) {
+  if (!d) return SPV_ERR_INVALID_ARG;
+  if (d->batch < 1 || d->grid_h < 1 || d->grid_w < 1 || d->block < 1 || d->radius < 0 || d->heads < 1)
+    return SPV_ERR_INVALID_ARG;
+  if (d->n_patch < 1 || d->n_patch > d->grid_h * d->grid_w) return SPV_ERR_INVALID_ARG;
+  if (!d->patch_pos && d->n_patch != d->grid_h * d->grid_w) return SPV_ERR_INVALID_ARG;
+  if (d->token_order != SPV_TOKENS_ROW_MAJOR && d->token_order != SPV_TOKENS_BLOCK_MAJOR)
+    return SPV_ERR_INVALID_ARG;
+  if (d->head_dim != HD) return SPV_ERR_UNSUPPORTED;
+  if (d->n_global < 1 || d->n_global > MAXG) return SPV_ERR_UNSUPPORTED;
+  if (d->stride_tok % 8 || d->stride_head % 8 || d->stride_b % 8) return SPV_ERR_ALIGNMENT;
+  if (d->stride_tok < HD || d->stride_head < HD) return SPV_ERR_INVALID_ARG;
+  return SPV_OK;
+}
+
+static size_t regroup_bytes(const spv_attn_desc* d) {
+  if (d->token_order == SPV_TOKENS_BLOCK_MAJOR) return 0;
+  return 3 * spv_align_up((size_t)d->batch * (d->n_global + d->n_patch) * d->heads * HD * 2, 256);
+}
+
+extern "C" int32_t spv_attn_workspace_size(const spv_attn_desc* d, size_t* bytes) {
+  int32_t st = validate_desc(d);
+  if (st != SPV_OK) return st;
+  if (!bytes) return SPV_ERR_INVALID_ARG;
+  *bytes = spv_attn_plan_bytes(d->batch, d->grid_h, d->grid_w, d->block, d->n_patch, d->token_order) +
+           regroup_bytes(d) + spv_attn_global_bytes(d->batch, d->n_global, d->heads, d->n_global + d->n_patch);
+  return SPV_OK;
+}
+
+extern "C" int32_t spatial_block_attention(spv_ctx* ctx, const spv_attn_desc* d, const void* q, const void* k,
+                                           const void* v, void* o, float* cls_scores, void* workspace,
+                                           size_t workspace_bytes, void* stream_) {
+  if (!ctx) return SPV_ERR_INVALID_ARG;
+  int32_t st = validate_desc(d);
+  if (st != SPV_OK) return st;
+  if (!q || !k || !v || !o) return SPV_ERR_INVALID_ARG;
+  if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15u) return SPV_ERR_ALIGNMENT;
+  size_t need;
+  spv_attn_workspace_size(d, &need);
+  if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255u)) return SPV_ERR_WORKSPACE;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  char* w = (char*)workspace;
+  const size_t plan_b = spv_attn_plan_bytes(d->batch, d->grid_h, d->grid_w, d->block, d->n_patch, d->token_order);
+  SpvAttnPlan plan;
+  st = spv_attn_plan_build(ctx, d->batch, d->grid_h, d->grid_w, d->block, d->radius, d->n_global, d->n_patch,
+                           d->patch_pos, d->token_order, w, plan_b, stream, &plan);
+  if (st != SPV_OK) return st;
+  w += plan_b;
+  const int n_tok = d->n_global + d->n_patch;
+  const float scale = d->softmax_scale != 0.f ? d->softmax_scale : 0.125f;
+  SpvAttnIO io;
+  io.heads = d->heads; io.scale = scale;
+  io.o = o; io.o_sb = d->stride_b; io.o_st = d->stride_tok; io.o_sh = d->stride_head;
+  // global-query rows read the caller's tensors directly (a dense row needs no grouping)
+  SpvAttnIO gio = io;
+  gio.q = q; gio.k = k; gio.v = v; gio.sb = d->stride_b; gio.st = d->stride_tok; gio.sh = d->stride_head;
+  gio.o_tok = nullptr;
+  if (d->token_order == SPV_TOKENS_ROW_MAJOR) {
+    const size_t one = spv_align_up((size_t)d->batch * n_tok * d->heads * HD * 2, 256);
+    __nv_bfloat16* qb = (__nv_bfloat16*)w; w += one;
+    __nv_bfloat16* kb = (__nv_bfloat16*)w; w += one;
+    __nv_bfloat16* vb = (__nv_bfloat16*)w; w += one;
+    const int64_t total = (int64_t)d->batch * n_tok * d->heads;
+    int64_t blocks = (total * 8 + 255) / 256;
+    const int64_t cap = (int64_t)ctx->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    attn_regroup<<<(unsigned)blocks, 256, 0, stream>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
+                                                      (const __nv_bfloat16*)v, d->stride_b, d->stride_tok,
+                                                      d->stride_head, qb, kb, vb, plan.bm_src, d->batch,
+                                                      d->n_global, d->n_patch, d->heads);
+    if ((st = spv_launch_ok(ctx)) != SPV_OK) return st;
+    io.q = qb; io.k = kb; io.v = vb;
+    io.st = (int64_t)d->heads * HD; io.sh = HD; io.sb = (int64_t)n_tok * d->heads * HD;
+    io.o_tok = plan.bm_src;
+  } else {
+    io.q = q; io.k = k; io.v = v; io.sb = d->stride_b; io.st = d->stride_tok; io.sh = d->stride_head;
+    io.o_tok = nullptr;
+  }
+  if ((st = spv_attn_run_patches(ctx, &plan, &io, stream)) != SPV_OK) return st;
+  return spv_attn_run_globals(ctx, &plan, &gio, cls_scores, nullptr, w,
+                              spv_attn_global_bytes(d->batch, d->n_global, d->heads, n_tok), stream);
+}

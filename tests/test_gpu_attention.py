@@ -1,0 +1,149 @@
+"""GPU parity of spatial_block_attention (Sec. 3.2) against the CPU oracle on the same seeded
+bf16 inputs.  Tolerance for bf16 outputs vs the fp32/fp64 oracle: max |err| <= 2e-2 and
+relative L2 <= 5e-3."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2601_12150_b200 as spv
+    c = spv.Context(0)
+    yield c
+    c.close()
+
+
+def _check(got, ref, max_abs=2e-2, rel_l2=5e-3):
+    err = got.astype(np.float64) - ref.astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.abs(err).max() <= max_abs, np.abs(err).max()
+    rel = np.linalg.norm(err) / np.linalg.norm(ref)
+    assert rel <= rel_l2, rel
+
+
+def _to_dev(ctx, a, packed=False):
+    """bf16 device tensor [B, N, h, 64]; `packed` lays q/k/v out as one [B, N, 3, h, 64] buffer."""
+    return torch.from_numpy(a).to(ctx.device).to(torch.bfloat16)
+
+
+def _run(ctx, q, k, v, gh, gw, b, r, G=1, patch_pos=None, order=0, packed=False, scores=True):
+    dev = ctx.device
+    if packed:
+        buf = torch.stack([torch.from_numpy(a) for a in (q, k, v)], dim=2).to(dev).to(torch.bfloat16)
+        dq, dk, dv = buf[:, :, 0], buf[:, :, 1], buf[:, :, 2]
+    else:
+        dq, dk, dv = (_to_dev(ctx, a) for a in (q, k, v))
+    pp = None if patch_pos is None else torch.from_numpy(np.ascontiguousarray(patch_pos, dtype=np.int32)).to(dev)
+    o, sc = ctx.spatial_block_attention(dq, dk, dv, gh, gw, b, r, n_global=G, patch_pos=pp,
+                                        token_order=order, want_scores=scores)
+    ctx.check()
+    return o.float().cpu().numpy(), None if sc is None else sc.cpu().numpy()
+
+
+def test_single_attention_op_28x28(ctx):
+    """785 tokens, 16 heads x 64, 7x7 blocks, 3x3 neighbourhood + CLS; and radius 3 == dense."""
+    q, k, v = synth.attention_qkv(0, 1, 785, 16, 64)
+    want, wsc = oracle.attention(q, k, v, 28, 28, 7, 1, want_scores=True)
+    got, gsc = _run(ctx, q, k, v, 28, 28, 7, 1)
+    _check(got, want)
+    assert np.abs(gsc - wsc).max() < 2e-4 * max(1.0, wsc.max() / 1e-2)
+    dense = oracle.dense_attention(q, k, v)
+    got3, _ = _run(ctx, q, k, v, 28, 28, 7, 3)
+    _check(got3, dense)
+    # the restriction is real: the sparse result differs from the dense one
+    assert np.abs(got - dense).max() > 5e-2
+
+
+@pytest.mark.parametrize("gh,gw,b,r,G,B,H", [
+    (16, 16, 8, 1, 1, 2, 2),      # exact tiles
+    (21, 13, 8, 1, 1, 1, 3),      # ragged edge blocks
+    (24, 40, 8, 2, 2, 1, 2),      # 5x5 neighbourhood, two global tokens
+    (12, 12, 2, 1, 1, 1, 2),      # small blocks: many blocks per query tile
+    (20, 20, 16, 0, 1, 1, 2),     # blocks larger than a tile (256 tokens), own block only
+    (9, 30, 4, 3, 1, 2, 1),       # wide neighbourhood
+])
+def test_geometries(ctx, gh, gw, b, r, G, B, H):
+    n = G + gh * gw
+    q, k, v = synth.attention_qkv(gh * 100 + gw, B, n, H, 64)
+    want, wsc = oracle.attention(q, k, v, gh, gw, b, r, n_global=G, want_scores=True)
+    got, gsc = _run(ctx, q, k, v, gh, gw, b, r, G=G, packed=True)
+    _check(got, want)
+    assert np.abs(gsc - wsc).max() < 1e-3
+
+
+def test_filtered_tokens_row_major_and_block_major(ctx):
+    gh, gw, b, r = 32, 24, 8, 1
+    rng = np.random.default_rng(5)
+    B, H = 2, 2
+    keep = np.stack([np.sort(rng.choice(gh * gw, size=400, replace=False)) for _ in range(B)]).astype(np.int32)
+    # image 1 loses every token of one block row to exercise empty blocks
+    alive = keep[1][(keep[1] // gw) // b != 1]
+    extra = np.setdiff1d(np.arange(gh * gw), keep[1])
+    extra = extra[(extra // gw) // b != 1][: 400 - alive.size]
+    keep[1] = np.sort(np.concatenate([alive, extra]))
+    n = 1 + 400
+    q, k, v = synth.attention_qkv(77, B, n, H, 64)
+    want, wsc = oracle.attention(q, k, v, gh, gw, b, r, patch_pos=keep, want_scores=True)
+    got, gsc = _run(ctx, q, k, v, gh, gw, b, r, patch_pos=keep)
+    _check(got, want)
+    assert np.abs(gsc - wsc).max() < 1e-3
+    # same tokens presented in block-major order
+    perm = np.stack([np.lexsort((keep[i], (keep[i] % gw) // b, (keep[i] // gw) // b)) for i in range(B)])
+    def reorder(a):
+        out = a.copy()
+        for i in range(B):
+            out[i, 1:] = a[i, 1 + perm[i]]
+        return out
+    keep_bm = np.stack([keep[i][perm[i]] for i in range(B)])
+    got_bm, gsc_bm = _run(ctx, reorder(q), reorder(k), reorder(v), gh, gw, b, r, patch_pos=keep_bm, order=1)
+    _check(got_bm, reorder(want))
+    for i in range(B):
+        assert np.abs(gsc_bm[i] - wsc[i][:, perm[i]]).max() < 1e-3
+
+
+def test_full_grid_block_major(ctx):
+    gh, gw, b, r = 20, 12, 8, 1
+    pos = np.arange(gh * gw)
+    perm = np.lexsort((pos, (pos % gw) // b, (pos // gw) // b))
+    q, k, v = synth.attention_qkv(9, 1, 1 + gh * gw, 2, 64)
+    want, _ = oracle.attention(q, k, v, gh, gw, b, r)
+    def reorder(a):
+        out = a.copy()
+        out[:, 1:] = a[:, 1 + perm]
+        return out
+    got, _ = _run(ctx, reorder(q), reorder(k), reorder(v), gh, gw, b, r, order=1, scores=False)
+    _check(got, reorder(want))
+
+
+def test_large_scores_and_argument_errors(ctx):
+    import paper_2601_12150_b200 as spv
+    # logits with a wide range exercise the running-maximum rescale
+    q, k, v = synth.attention_qkv(21, 1, 1 + 256, 2, 64, std=2.5)
+    want, _ = oracle.attention(q, k, v, 16, 16, 8, 1)
+    got, _ = _run(ctx, q, k, v, 16, 16, 8, 1)
+    _check(got, want, max_abs=4e-2)
+    dq = torch.zeros((1, 17, 2, 32), dtype=torch.bfloat16, device=ctx.device)
+    with pytest.raises(spv.SpvError) as e:
+        ctx.spatial_block_attention(dq, dq, dq, 4, 4, 2, 1)
+    assert e.value.status == spv.ERR_UNSUPPORTED
+    dq = torch.zeros((1, 17, 2, 64), dtype=torch.bfloat16, device=ctx.device)
+    with pytest.raises(spv.SpvError):
+        ctx.spatial_block_attention(dq, dq, dq, 5, 4, 2, 1)       # n_patch != H*W without positions
+
+
+def test_sampled_rows_at_full_size(ctx):
+    """ViT-L/16 at 2048^2 geometry (128x128 grid, 16385 tokens), sampled query rows vs the oracle."""
+    gh = gw = 128
+    q, k, v = synth.attention_qkv(3, 1, 1 + gh * gw, 4, 64)
+    got, gsc = _run(ctx, q, k, v, gh, gw, 8, 1, packed=True)
+    rng = np.random.default_rng(0)
+    rows = np.unique(np.concatenate([[0, 1, gh * gw], rng.integers(1, 1 + gh * gw, size=300)])).astype(np.int32)
+    want, wsc = oracle.attention(q, k, v, gh, gw, 8, 1, rows=rows, want_scores=True)
+    _check(got[:, rows], want[:, rows])
+    assert np.abs(gsc - wsc).max() < 1e-3

@@ -24,7 +24,8 @@ def _bf16(dev, a):
 
 def _check(got, ref, max_abs=2e-2, rel_l2=5e-3):
     err = got.astype(np.float64) - ref.astype(np.float64)
-    assert np.abs(err).max() <= max_abs, np.abs(err).max()
+    # bf16 output: the absolute bound scales with the magnitude above 1 (one bf16 ulp at |x| is |x|/128)
+    assert (np.abs(err) <= max_abs * np.maximum(1.0, np.abs(ref))).all(), np.abs(err).max()
     assert np.linalg.norm(err) / max(np.linalg.norm(ref), 1e-30) <= rel_l2
 
 
@@ -84,7 +85,7 @@ def test_gemm_epilogues(ctx, epi):
         ctx.gemm_bf16(A, W, out, spv.EPI_BIAS_MUL, bias=Bv, aux=_bf16(dev, aux))
         ref = lin * aux
     ctx.check()
-    _check(out.float().cpu().numpy(), ref, max_abs=4e-2)
+    _check(out.float().cpu().numpy(), ref)
 
 
 @pytest.mark.parametrize("rows,dim", [(5, 64), (4097, 1024), (1000, 1536), (33, 2304)])
