@@ -54,6 +54,9 @@ int32_t spv_destroy(spv_ctx* ctx);
 const char* spv_status_string(int32_t status);
 /* Synchronise `stream`, then return and clear the latched device-side status. */
 int32_t spv_check(spv_ctx* ctx, void* stream);
+/* Site code of the bounded wait that the last failing spv_check() reported (0 = none): the
+ * kernel and barrier that gave up, for diagnosis. */
+uint32_t spv_last_wait_site(const spv_ctx* ctx);
 /* Number of kernels this context has launched so far (host counter, for accounting). */
 int64_t spv_launch_count(const spv_ctx* ctx);
 

@@ -17,7 +17,7 @@ MLP_GELU, MLP_SWIGLU = 0, 1
 ATTN_DENSE, ATTN_SPARSE = 0, 1
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_SILU, EPI_BIAS_MUL, EPI_BIAS_SCALE_RESID, EPI_BIAS_ADDROW = range(6)
 
-EXPORTS = ["spv_create", "spv_destroy", "spv_status_string", "spv_check", "spv_launch_count",
+EXPORTS = ["spv_create", "spv_destroy", "spv_status_string", "spv_check", "spv_last_wait_site", "spv_launch_count",
            "spv_attn_workspace_size", "spatial_block_attention",
            "spv_filter_keep_count", "spv_filter_workspace_size", "cls_score_topk_filter",
            "spv_vit_workspace_size", "vit_forward", "spv_gemm_bf16", "spv_layernorm"]
@@ -88,6 +88,8 @@ def lib():
         L.spv_status_string.argtypes = [C.c_int32]
         L.spv_launch_count.restype = C.c_int64
         L.spv_launch_count.argtypes = [C.c_void_p]
+        L.spv_last_wait_site.restype = C.c_uint32
+        L.spv_last_wait_site.argtypes = [C.c_void_p]
         L.spv_create.argtypes = [C.POINTER(C.c_void_p), C.c_int32]
         L.spv_destroy.argtypes = [C.c_void_p]
         L.spv_check.argtypes = [C.c_void_p, C.c_void_p]
@@ -169,7 +171,10 @@ class Context:
         return self._ws
 
     def check(self, stream=None):
-        _raise(lib().spv_check(self.handle, _stream(stream)), "spv_check")
+        st = lib().spv_check(self.handle, _stream(stream))
+        if st == ERR_TIMEOUT:
+            raise SpvError(st, "spv_check (wait site 0x%x)" % lib().spv_last_wait_site(self.handle))
+        _raise(st, "spv_check")
 
     def launch_count(self):
         return int(lib().spv_launch_count(self.handle))

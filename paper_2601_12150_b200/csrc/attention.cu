@@ -547,18 +547,26 @@ __global__ void __launch_bounds__(256) attn_global_partial(const __nv_bfloat16* 
   for (int i = threadIdx.x; i < GCH; i += 256) s_s[i] = -INFINITY;
   __syncthreads();
   float lmax = -INFINITY;
-  for (int kk = k0 + grp; kk < k1; kk += 32) {
-    float kf[8];
-    unpack8(__ldg(reinterpret_cast<const uint4*>(k + b * sb + (int64_t)kk * st + (int64_t)h * sh) + sub), kf);
+  // the trip count is the same for every lane (the shuffles name the whole warp); keys past the
+  // end of the chunk are predicated off
+  for (int kk0 = k0; kk0 < k1; kk0 += 32) {
+    const int kk = kk0 + grp;
+    const bool live = kk < k1;
     float d = 0.f;
+    if (live) {
+      float kf[8];
+      unpack8(__ldg(reinterpret_cast<const uint4*>(k + b * sb + (int64_t)kk * st + (int64_t)h * sh) + sub), kf);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) d = fmaf(qf[i], kf[i], d);
+      for (int i = 0; i < 8; ++i) d = fmaf(qf[i], kf[i], d);
+    }
     d += __shfl_xor_sync(0xffffffffu, d, 1);
     d += __shfl_xor_sync(0xffffffffu, d, 2);
     d += __shfl_xor_sync(0xffffffffu, d, 4);
     d *= scale;
-    if (sub == 0) s_s[kk - k0] = d;
-    lmax = fmaxf(lmax, d);
+    if (live) {
+      if (sub == 0) s_s[kk - k0] = d;
+      lmax = fmaxf(lmax, d);
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) lmax = fmaxf(lmax, __shfl_xor_sync(0xffffffffu, lmax, o));

@@ -23,6 +23,7 @@ struct spv_ctx {
   uint32_t* d_status;            // device status word: 0 = ok, else first failing site code
   spv_encode_tiled_fn encode_tiled;
   int64_t launches;
+  uint32_t last_site;            // site code read by the last failing spv_check
 };
 
 #define SPV_CUDA_OK(expr)                         \
@@ -92,11 +93,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Bounded wait: gives up after SPV_WAIT_LIMIT_NS of polling, latches `site` in the status word
-// and in the CTA's abort flag so that every later wait of the CTA returns at once.  The kernel
+// and in the CTA's abort flag so that every later wait of the CTA (and, through the status word,
+// of every other CTA of the grid) returns at once.  The kernel
 // then runs to its normal end (its loops are bounded by tile counts), releases TMEM and exits;
 // the host reads the status through spv_check().
 #ifndef SPV_WAIT_LIMIT_NS
-#define SPV_WAIT_LIMIT_NS 2000000000ull
+#define SPV_WAIT_LIMIT_NS 1000000000ull
 #endif
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
@@ -110,6 +112,8 @@ static __device__ __noinline__ void mbar_wait_slow(uint64_t* bar, uint32_t parit
     if (mbar_try_wait(bar, parity)) return;
     if ((it & 63u) == 63u) {
       if (*abort_flag) return;
+      // another CTA already gave up: do not wait out a second limit here
+      if (*reinterpret_cast<volatile uint32_t*>(status) != 0u) { *abort_flag = 1; return; }
       if (global_ns() - t0 > SPV_WAIT_LIMIT_NS) break;
     }
   }

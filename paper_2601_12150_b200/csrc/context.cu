@@ -59,11 +59,14 @@ extern "C" int32_t spv_check(spv_ctx* ctx, void* stream) {
   uint32_t st = 0;
   SPV_CUDA_OK(cudaMemcpy(&st, ctx->d_status, sizeof(st), cudaMemcpyDeviceToHost));
   if (st != 0) {
+    ctx->last_site = st;
     cudaMemset(ctx->d_status, 0, sizeof(st));
     return SPV_ERR_TIMEOUT;
   }
   return SPV_OK;
 }
+
+extern "C" uint32_t spv_last_wait_site(const spv_ctx* ctx) { return ctx ? ctx->last_site : 0u; }
 
 extern "C" int64_t spv_launch_count(const spv_ctx* ctx) { return ctx ? ctx->launches : 0; }
 

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def _declared():
     text = open(os.path.join(ROOT, "include", "spatvit.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = re.findall(r"\b(?:int32_t|int64_t|const char\*)\s+(\w+)\s*\(", text)
+    names = re.findall(r"\b(?:int32_t|int64_t|uint32_t|const char\*)\s+(\w+)\s*\(", text)
     return sorted(set(names))
 
 
