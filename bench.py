@@ -1,0 +1,421 @@
+#!/usr/bin/env python
+"""Throughput of the large-resolution ViT inference path on B200: images/s of ViT-L/16 at
+2048x2048 with neighbouring-block sparse attention and the CLS-score token filter.
+
+One step = one vit_forward over one batch of synthetic tissue-like images (patch embedding, 24
+blocks with sparse attention, the filter after block 4, final LayerNorm).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
+    python bench.py --impl reference ...     # the CPU oracle on a bounded sample of the workload
+
+Prints ONE JSON line.  `value` is measured with the inputs resident in device memory; `e2e`
+includes the pinned-host -> device copy of the images and the device -> host read of the output
+tokens in every step.  `roofline` describes the kernel class with the largest share of the step,
+`breakdown` every class, `cpu_baseline` the oracle timed on this host's cores.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+METRIC = "ViT-L/16 images/s at 2048x2048 (sparse attention + token filter)"
+
+WORKLOADS = {
+    # name: (arch, image side, batch, block, radius, filter_layer, keep, weight seed, image seed)
+    "vitl16_2048_b4_sparse_filter": ("l16", 2048, 4, 8, 1, 4, 0.5, 2, 6),
+    "vitl16_2048_b4_sparse": ("l16", 2048, 4, 8, 1, 0, 1.0, 2, 6),
+    "vitl16_1024_b1_sparse_filter": ("l16", 1024, 1, 8, 1, 4, 0.6, 2, 3),
+    "vitl16_1024_b4_sparse_filter": ("l16", 1024, 4, 8, 1, 4, 0.5, 2, 6),
+    "vitl16_448_b4_sparse_filter": ("l16", 448, 4, 8, 1, 4, 0.5, 2, 6),
+}
+DEFAULT_WORKLOAD = "vitl16_2048_b4_sparse_filter"
+
+
+def workload_config(name):
+    arch_name, side, batch, block, radius, fl, keep, wseed, iseed = WORKLOADS[name]
+    arch = synth.vit_l16() if arch_name == "l16" else synth.vit_g14()
+    grid = side // arch["patch"]
+    cfg = dict(arch, attn_mode=synth.ATTN_SPARSE, block=block, radius=radius, filter_layer=fl, keep_ratio=keep)
+    return dict(name=name, arch=arch, cfg=cfg, side=side, grid=grid, batch=batch, wseed=wseed, iseed=iseed)
+
+
+# --------------------------------------------------------------------------------------------
+# algorithmic work (counting only; none of the method's arithmetic)
+# --------------------------------------------------------------------------------------------
+def attention_pairs(grid_h, grid_w, block, radius, n_global, positions=None):
+    """(patch-query pairs incl. global key columns, global-query pairs) of one image and head."""
+    pos = np.arange(grid_h * grid_w) if positions is None else np.asarray(positions)
+    nby, nbx = -(-grid_h // block), -(-grid_w // block)
+    cnt = np.zeros((nby, nbx), dtype=np.int64)
+    np.add.at(cnt, ((pos // grid_w) // block, (pos % grid_w) // block), 1)
+    integ = np.zeros((nby + 1, nbx + 1), dtype=np.int64)
+    integ[1:, 1:] = cnt.cumsum(0).cumsum(1)
+    by, bx = np.meshgrid(np.arange(nby), np.arange(nbx), indexing="ij")
+    y0, y1 = np.maximum(by - radius, 0), np.minimum(by + radius, nby - 1) + 1
+    x0, x1 = np.maximum(bx - radius, 0), np.minimum(bx + radius, nbx - 1) + 1
+    nsum = integ[y1, x1] - integ[y0, x1] - integ[y1, x0] + integ[y0, x0]
+    n_p = int(cnt.sum())
+    return int((cnt * nsum).sum()) + n_p * n_global, n_global * (n_global + n_p)
+
+
+def forward_flops(wl, kept_positions):
+    """Useful FLOP of one step: GEMMs (2MNK) and attention (4*64 per allowed pair and head)."""
+    a, c, g, B = wl["arch"], wl["cfg"], wl["grid"], wl["batch"]
+    D, HID, H, G = a["dim"], a["mlp_hidden"], a["heads"], a["n_global"]
+    n0 = G + g * g
+    per_tok = 2 * D * (3 * D) + 2 * D * D + 2 * D * HID * (3 if a["mlp_kind"] == synth.MLP_SWIGLU else 2)
+    gemm = 2.0 * B * g * g * (3 * a["patch"] ** 2) * D
+    attn_patch = attn_glob = 0.0
+    fl = c["filter_layer"]
+    pre_p, pre_g = attention_pairs(g, g, c["block"], c["radius"], G)
+    n_pre = a["layers"] if fl == 0 else fl
+    gemm += n_pre * B * n0 * per_tok
+    attn_patch += n_pre * B * 4.0 * 64 * H * pre_p
+    attn_glob += n_pre * B * 4.0 * 64 * H * pre_g
+    for b in range(B if fl > 0 else 0):
+        pp, pg = attention_pairs(g, g, c["block"], c["radius"], G, kept_positions[b])
+        n_post = a["layers"] - fl
+        gemm += n_post * (G + len(kept_positions[b])) * per_tok
+        attn_patch += n_post * 4.0 * 64 * H * pp
+        attn_glob += n_post * 4.0 * 64 * H * pg
+    return dict(gemm=gemm, attn_patch=attn_patch, attn_global=attn_glob)
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=float(p["hbm_gbs"]), tensor=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    tensor_burst=float(p["bf16_tflops"]), source="measured")
+    return dict(hbm=6650.0, tensor=1400.0, tensor_burst=1590.0, source="fallback")
+
+
+# --------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle leg
+# --------------------------------------------------------------------------------------------
+def oracle_sample(wl, rows, seed=11):
+    """Time the oracle, as it stands, on a bounded sample of the workload and extrapolate to
+    images/s.  Sample: `rows` token rows of every per-token operation of one block (LayerNorm,
+    QKV / out / MLP linears, activation, residual adds) plus `rows` query rows of the sparse
+    attention against all keys, once at the full token count and once at the post-filter count
+    (a spatially coherent kept set); plus `rows` rows of the patch-embedding linear.  Every cost
+    is linear in rows at a fixed token count, so
+      T_image = N (t_embed + f (t_tok + t_attn_full)) + N' (L - f) (t_tok + t_attn_kept)  per row.
+    """
+    import oracle
+    a, c, g = wl["arch"], wl["cfg"], wl["grid"]
+    D, HID, H, G, L = a["dim"], a["mlp_hidden"], a["heads"], a["n_global"], a["layers"]
+    rng = np.random.Generator(np.random.PCG64(seed))
+    one = dict(a, layers=1)
+    w = synth.vit_weights(wl["wseed"], one, 2, 2, pos_base=2)
+    lw = w["layers"][0]
+    np0 = g * g
+    n0 = G + np0
+    fl = c["filter_layer"]
+    k = oracle.keep_count(np0, c["keep_ratio"]) if fl > 0 else np0
+    n1 = G + k
+    rows = min(rows, n1)
+    x = rng.standard_normal((rows, D), dtype=np.float32)
+    cols = synth.round_bf16(rng.standard_normal((rows, 3 * a["patch"] ** 2), dtype=np.float32))
+    t = {}
+    t0 = time.perf_counter()
+    oracle.linear(cols, w["w_pe"], w["b_pe"])
+    t["embed"] = time.perf_counter() - t0
+
+    def per_token():
+        h = oracle.layernorm(x, lw["ln1_g"], lw["ln1_b"], a["ln_eps"])
+        oracle.linear(h, lw["w_qkv"], lw["b_qkv"])
+        y = x + lw.get("ls1", 1.0) * oracle.linear(h, lw["w_o"], lw["b_o"])
+        h = oracle.layernorm(y, lw["ln2_g"], lw["ln2_b"], a["ln_eps"])
+        u = oracle.linear(h, lw["w_fc1"], lw["b_fc1"])
+        if a["mlp_kind"] == synth.MLP_SWIGLU:
+            u = oracle.silu_mul_n(u, oracle.linear(h, lw["w_fc3"], lw["b_fc3"]))
+        else:
+            u = oracle.gelu_n(u)
+        return y + lw.get("ls2", 1.0) * oracle.linear(u, lw["w_fc2"], lw["b_fc2"])
+
+    t0 = time.perf_counter()
+    per_token()
+    t["tok"] = time.perf_counter() - t0
+
+    def attn(n_tok, positions):
+        q, kk, v = synth.attention_qkv(seed + n_tok, 1, n_tok, H, D // H)
+        qrows = np.sort(rng.choice(n_tok, size=rows, replace=False)).astype(np.int32)
+        pp = None if positions is None else positions[None].astype(np.int32)
+        t0 = time.perf_counter()
+        oracle.attention(q, kk, v, g, g, c["block"], c["radius"], n_global=G, patch_pos=pp, rows=qrows)
+        return time.perf_counter() - t0
+
+    t["attn_full"] = attn(n0, None)
+    if fl > 0:
+        bg = synth.background_mask(rng, g, g, 1.0 - k / np0).reshape(-1)
+        kept = np.flatnonzero(~bg)[:k]
+        if kept.size < k:
+            kept = np.sort(np.concatenate([kept, np.flatnonzero(bg)[:k - kept.size]]))
+        t["attn_kept"] = attn(n1, kept)
+    else:
+        t["attn_kept"] = t["attn_full"]
+    f = fl if fl > 0 else L
+    t_image = (n0 * (t["embed"] + f * (t["tok"] + t["attn_full"])) + n1 * (L - f) * (t["tok"] + t["attn_kept"])) / rows
+    total = sum(t.values())
+    return dict(images_per_s=1.0 / t_image, sample_seconds=total, rows=rows, cores=oracle.num_threads(),
+                parts={k_: round(v_, 4) for k_, v_ in t.items()})
+
+
+def run_reference(args, wl, rank):
+    if rank != 0:
+        return
+    rows = 512
+    for _ in range(args.warmup):
+        oracle_sample(wl, rows)
+    times, rates, last = [], [], None
+    for _ in range(args.steps):
+        last = oracle_sample(wl, rows)
+        times.append(last["sample_seconds"])
+        rates.append(last["images_per_s"])
+    value = statistics.mean(rates)
+    sample = (f"{rows} token rows of each per-token op of one block + {rows} attention query rows at the full and "
+              f"post-filter token counts + {rows} patch-embedding rows of one {wl['side']}x{wl['side']} image, "
+              "extrapolated linearly in rows to a whole image")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl["name"], "l2": "inputs larger than L2"},
+        "cpu_baseline": {"value": value, "unit": "images/s", "cores": last["cores"], "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+def run_gpu(args, wl, rank, world):
+    import torch
+    import torch.distributed as dist
+    import paper_2601_12150_b200 as spv
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    ctx = spv.Context(local)
+    a, c, g, B = wl["arch"], wl["cfg"], wl["grid"], wl["batch"]
+    side = wl["side"]
+
+    w = synth.vit_weights(wl["wseed"], a, g, g)
+    dw = ctx.make_vit_weights(w)
+    del w
+    img_host = torch.from_numpy(synth.tissue_batch(wl["iseed"] + rank, B, side, side,
+                                                   background_range=(0.3, 0.6))).pin_memory()
+    img = img_host.to(dev)
+    k = spv.filter_keep_count(g * g, c["keep_ratio"]) if c["filter_layer"] > 0 else g * g
+    out = torch.empty((B, a["n_global"] + k, a["dim"]), dtype=torch.bfloat16, device=dev)
+    out_host = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def step():
+        return ctx.vit_forward(c, dw, img, g, g, out=out)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    torch.cuda.reset_peak_memory_stats()
+    n_warm = max(args.warmup, 1) if args.quick else max(args.warmup, 3)
+    for _ in range(n_warm):
+        _, kept = step()
+    ctx.check()
+    kept_host = kept.cpu().numpy() if kept is not None else None
+
+    # ---- timed region: device-resident inputs, per-class event timing on
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    barrier()
+    sampler.start()
+    launches0 = ctx.launch_count()
+    ctx.profile(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = ctx.launch_count() - launches0
+    prof = ctx.profile_read()
+    ctx.profile(False)
+    ctx.check()
+    clocks = sampler.stop()
+    peak_bytes = torch.cuda.max_memory_allocated()
+
+    # ---- end to end: pinned host images in, output tokens back to the host, every step
+    def e2e_step():
+        img.copy_(img_host, non_blocking=True)
+        step()
+        out_host.copy_(out, non_blocking=True)
+
+    ms_e2e = float("nan")
+    if not args.quick:
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for _ in range(args.steps):
+            e2e_step()
+        f1.record(stream)
+        barrier()
+        ms_e2e = f0.elapsed_time(f1)
+        ctx.check()
+
+    if world > 1:
+        tt = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = tt.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    images = B * args.steps * world
+    value = images / (ms * 1e-3)
+    fl = forward_flops(wl, kept_host)
+    steps = args.steps
+    tot_ms = sum(v["ms"] for v in prof.values()) or 1.0
+    brk = {}
+    for name, v in prof.items():
+        if v["launches"] == 0:
+            continue
+        e = dict(launches_per_step=v["launches"] / steps, ms_per_step=v["ms"] / steps, share=v["ms"] / tot_ms)
+        sec = v["ms"] * 1e-3
+        if name == "gemm":
+            e.update(bound="tensor", achieved=v["work"] / sec / 1e12, unit="TFLOP/s", peak=pk["tensor"])
+        elif name == "attn_patch":
+            e.update(bound="tensor", achieved=fl["attn_patch"] * steps / sec / 1e12, unit="useful TFLOP/s",
+                     peak=pk["tensor"])
+        elif name in ("layernorm", "filter_gather", "filter_select"):
+            e.update(bound="hbm", achieved=v["work"] / sec / 1e9, unit="GB/s", peak=pk["hbm"])
+        if "achieved" in e:
+            e["frac"] = e["achieved"] / e["peak"]
+        brk[name] = e
+    top = max(brk, key=lambda n: brk[n]["share"])
+    roof = {"kernel": top, "bound": brk[top].get("bound"), "achieved": brk[top].get("achieved"),
+            "peak": brk[top].get("peak"), "unit": "TFLOP/s" if brk[top].get("bound") == "tensor" else "GB/s",
+            "frac": brk[top].get("frac"), "traffic": None,
+            "peak_source": f"of {pk['source']} (sustained bf16 figure: the kernel is timed inside a long step)"}
+    total_flops = fl["gemm"] + fl["attn_patch"] + fl["attn_global"]
+    line = {
+        "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": steps, "warmup": n_warm,
+        "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl["name"], "image": f"{side}x{side}", "batch_per_gpu": B, "grid": f"{g}x{g}",
+                   "tokens": a["n_global"] + g * g, "block": c["block"], "radius": c["radius"],
+                   "filter_layer": c["filter_layer"], "keep_ratio": c["keep_ratio"], "kept": k,
+                   "parallelism": "replicas" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2 (activations of one step exceed 126 MB)"},
+        "clocks": clocks, "gpu_launches": launches,
+        "e2e": {"value": images / (ms_e2e * 1e-3), "unit": "images/s",
+                "h2d_bytes_per_step": img_host.numel() * 4, "d2h_bytes_per_step": out_host.numel() * 2},
+        "roofline": roof, "breakdown": brk,
+        "useful_tflops": total_flops * steps * world / (ms * 1e-3) / 1e12,
+        "peak_hbm_bytes": peak_bytes,
+    }
+    if world == 1 and not args.no_cpu and not args.quick:
+        cb = oracle_sample(wl, args.cpu_rows)
+        line["cpu_baseline"] = {
+            "value": cb["images_per_s"], "unit": "images/s", "cores": cb["cores"], "kind": "oracle",
+            "sample": (f"{cb['rows']} token rows of each per-token op of one block, {cb['rows']} attention query "
+                       f"rows at the full and post-filter token counts and {cb['rows']} patch-embedding rows of one "
+                       f"image ({cb['sample_seconds']:.1f} s of CPU work), extrapolated linearly in rows"),
+            "parts_s": cb["parts"]}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--cpu-rows", type=int, default=16384, help="rows of the CPU-oracle sample")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--quick", action="store_true",
+                    help="profiling aid: exactly --warmup warm-up steps, no end-to-end and no CPU leg")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    wl = workload_config(args.workload)
+    if args.impl == "reference":
+        run_reference(args, wl, rank)
+    else:
+        run_gpu(args, wl, rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -229,6 +229,33 @@ int32_t spv_gemm_bf16(spv_ctx* ctx, const spv_gemm_desc* desc, const void* a, co
 int32_t spv_layernorm(spv_ctx* ctx, const float* x, int64_t rows, int32_t dim, const float* gamma,
                       const float* beta, float eps, void* y, const int32_t* out_row, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Per-kernel-class device timing (CUDA events recorded on the launch stream around every
+ * launch while enabled; a few hundred nanoseconds per launch).  Off by default.
+ * ---------------------------------------------------------------------------------------- */
+enum {
+  SPV_K_GEMM = 0,          /* tcgen05 GEMMs (QKV, out-proj, MLP, patch embedding)              */
+  SPV_K_ATTN_PATCH = 1,    /* sparse-attention flash kernel, patch queries                     */
+  SPV_K_ATTN_GLOBAL = 2,   /* global-token rows and CLS->patch scores                          */
+  SPV_K_ATTN_PLAN = 3,     /* block offsets / query tiles / regrouping copy                    */
+  SPV_K_LAYERNORM = 4,
+  SPV_K_FILTER_SELECT = 5, /* head mean + ranking                                              */
+  SPV_K_FILTER_GATHER = 6, /* compaction copy of the surviving rows                            */
+  SPV_K_MISC = 7,          /* im2col, position tables, output row map                          */
+  SPV_K_COUNT = 8
+};
+typedef struct {
+  int64_t launches;  /* timed launch groups of this class                                      */
+  double ms;         /* summed device time                                                     */
+  double work;       /* summed algorithmic work: FLOP for SPV_K_GEMM, bytes for LayerNorm and
+                        the filter kernels, 0 where the caller has to count it                 */
+} spv_kernel_stat;
+/* enable != 0: start timing (and clear the accumulated figures); 0: stop. */
+int32_t spv_profile_enable(spv_ctx* ctx, int32_t enable);
+/* Wait for the recorded events, add them into `out` (host array of SPV_K_COUNT entries) and
+ * clear the record. */
+int32_t spv_profile_read(spv_ctx* ctx, spv_kernel_stat* out);
+
 #ifdef __cplusplus
 }
 #endif

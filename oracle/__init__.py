@@ -53,6 +53,8 @@ def lib():
         _lib.spvo_silu.restype = C.c_float
         _lib.spvo_silu.argtypes = [C.c_float]
         _lib.spvo_keep_count.argtypes = [C.c_int32, C.c_double]
+        _lib.spvo_gelu_n.restype = None
+        _lib.spvo_silu_mul_n.restype = None
         _lib.spvo_layernorm.restype = None
         _lib.spvo_linear.restype = None
     return _lib
@@ -180,6 +182,22 @@ def gelu(x):
 
 def silu(x):
     return float(lib().spvo_silu(float(x)))
+
+
+def gelu_n(a):
+    """Exact (erf) GELU over an array."""
+    a = _f32(a)
+    y = np.empty_like(a)
+    lib().spvo_gelu_n(_ptr(a), C.c_int64(a.size), _ptr(y))
+    return y
+
+
+def silu_mul_n(a, b):
+    """silu(a) * b over arrays (the SwiGLU gate)."""
+    a, b = _f32(a), _f32(b)
+    y = np.empty_like(a)
+    lib().spvo_silu_mul_n(_ptr(a), _ptr(b), C.c_int64(a.size), _ptr(y))
+    return y
 
 
 def vit_forward(cfg, weights, image, grid_h, grid_w, forced_keep=None, tap_layer=None):

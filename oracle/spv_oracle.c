@@ -277,6 +277,13 @@ void spvo_linear(const float* x, int64_t rows, int32_t in_dim, int32_t out_dim,
 float spvo_gelu(float x) { return (float)(0.5 * (double)x * (1.0 + erf((double)x / sqrt(2.0)))); }
 float spvo_silu(float x) { return (float)((double)x / (1.0 + exp(-(double)x))); }
 
+void spvo_gelu_n(const float* a, int64_t n, float* y) {
+  for (int64_t i = 0; i < n; ++i) y[i] = spvo_gelu(a[i]);
+}
+void spvo_silu_mul_n(const float* a, const float* b, int64_t n, float* y) {
+  for (int64_t i = 0; i < n; ++i) y[i] = spvo_silu(a[i]) * b[i];
+}
+
 int32_t spvo_vit_forward(const spvo_vit_config* c, const spvo_vit_weights* w,
                          const float* image, int32_t batch, int32_t gh, int32_t gw,
                          float* out_tokens, int32_t* kept_idx,

@@ -129,6 +129,9 @@ void spvo_linear(const float* x, int64_t rows, int32_t in_dim, int32_t out_dim,
                  const float* w /*[out,in]*/, const float* bias, float* y);
 float spvo_gelu(float x);
 float spvo_silu(float x);
+/* The same two activations over arrays: y[i] = gelu(a[i]);  y[i] = silu(a[i]) * b[i]. */
+void spvo_gelu_n(const float* a, int64_t n, float* y);
+void spvo_silu_mul_n(const float* a, const float* b, int64_t n, float* y);
 
 int32_t spvo_num_threads(void);
 

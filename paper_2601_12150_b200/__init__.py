@@ -20,7 +20,8 @@ EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_SILU, EPI_BIAS_MUL, EPI_BIAS_SCALE_RESID, EPI_
 EXPORTS = ["spv_create", "spv_destroy", "spv_status_string", "spv_check", "spv_last_wait_site", "spv_launch_count",
            "spv_attn_workspace_size", "spatial_block_attention",
            "spv_filter_keep_count", "spv_filter_workspace_size", "cls_score_topk_filter",
-           "spv_vit_workspace_size", "vit_forward", "spv_gemm_bf16", "spv_layernorm"]
+           "spv_vit_workspace_size", "vit_forward", "spv_gemm_bf16", "spv_layernorm",
+           "spv_profile_enable", "spv_profile_read"]
 
 
 class SpvError(RuntimeError):
@@ -63,6 +64,14 @@ class VitWeights(C.Structure):
     _fields_ = [("w_pe", C.c_void_p), ("b_pe", C.c_void_p), ("cls", C.c_void_p),
                 ("pos", C.c_void_p), ("lnf_g", C.c_void_p), ("lnf_b", C.c_void_p),
                 ("layer", C.c_void_p)]
+
+
+KERNEL_CLASSES = ["gemm", "attn_patch", "attn_global", "attn_plan", "layernorm", "filter_select",
+                  "filter_gather", "misc"]
+
+
+class KernelStat(C.Structure):
+    _fields_ = [("launches", C.c_int64), ("ms", C.c_double), ("work", C.c_double)]
 
 
 class GemmDesc(C.Structure):
@@ -109,6 +118,8 @@ def lib():
                                     C.c_void_p]
         L.spv_layernorm.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p,
                                     C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.spv_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+        L.spv_profile_read.argtypes = [C.c_void_p, C.POINTER(KernelStat)]
         _lib = L
     return _lib
 
@@ -178,6 +189,17 @@ class Context:
 
     def launch_count(self):
         return int(lib().spv_launch_count(self.handle))
+
+    def profile(self, enable=True):
+        """Start (and clear) or stop the per-kernel-class event timing."""
+        _raise(lib().spv_profile_enable(self.handle, 1 if enable else 0), "spv_profile_enable")
+
+    def profile_read(self):
+        """{class: dict(launches, ms, work)} accumulated since the last read; waits for the events."""
+        arr = (KernelStat * len(KERNEL_CLASSES))()
+        _raise(lib().spv_profile_read(self.handle, arr), "spv_profile_read")
+        return {n: dict(launches=int(a.launches), ms=float(a.ms), work=float(a.work))
+                for n, a in zip(KERNEL_CLASSES, arr)}
 
     # -- Sec. 3.3 ---------------------------------------------------------------------------
     def cls_score_topk_filter(self, scores, tokens_in=None, n_global=1, keep_ratio=0.5,

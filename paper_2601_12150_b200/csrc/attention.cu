@@ -735,6 +735,7 @@ int32_t spv_attn_plan_build(spv_ctx* ctx, int32_t batch, int32_t grid_h, int32_t
   p.bm_src = (int32_t*)take((size_t)batch * n_patch * 4);
   p.tiles = (int4*)take((size_t)batch * p.tiles_per_image * sizeof(int4));
   const dim3 sgrid((p.nseg + 255) / 256, batch);
+  SpvProfScope prof(ctx, SPV_K_ATTN_PLAN, stream);
   attn_plan_segments<<<sgrid, 256, 0, stream>>>(p, patch_pos, token_order);
   attn_plan_scan<<<batch, 1024, 0, stream>>>(p);
   attn_plan_fill<<<sgrid, 256, 0, stream>>>(p);
@@ -764,6 +765,7 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   pp.scale_log2 = io->scale * 1.4426950408889634f;
   pp.status = ctx->d_status;
   const dim3 grid(plan->tiles_per_image, io->heads, plan->batch);
+  SpvProfScope prof(ctx, SPV_K_ATTN_PATCH, stream);
   attn_patch_kernel<<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, pp);
   return spv_launch_ok(ctx);
 }
@@ -785,6 +787,7 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   float* logits = (float*)w; w += spv_align_up(rows * n_tok * 4, 256);
   float* part_ml = (float*)w; w += spv_align_up(rows * chunks * 2 * 4, 256);
   float* part_o = (float*)w;
+  SpvProfScope prof(ctx, SPV_K_ATTN_GLOBAL, stream);
   attn_global_partial<<<dim3(chunks, io->heads, B * G), 256, 0, stream>>>(
       (const __nv_bfloat16*)io->q, (const __nv_bfloat16*)io->k, (const __nv_bfloat16*)io->v, io->sb, io->st, io->sh,
       n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks);
@@ -863,6 +866,7 @@ extern "C" int32_t spatial_block_attention(spv_ctx* ctx, const spv_attn_desc* d,
     int64_t blocks = (total * 8 + 255) / 256;
     const int64_t cap = (int64_t)ctx->sm_count * 16;
     if (blocks > cap) blocks = cap;
+    SpvProfScope prof(ctx, SPV_K_ATTN_PLAN, stream);
     attn_regroup<<<(unsigned)blocks, 256, 0, stream>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                                       (const __nv_bfloat16*)v, d->stride_b, d->stride_tok,
                                                       d->stride_head, qb, kb, vb, plan.bm_src, d->batch,

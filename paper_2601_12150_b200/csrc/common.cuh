@@ -24,6 +24,18 @@ struct spv_ctx {
   spv_encode_tiled_fn encode_tiled;
   int64_t launches;
   uint32_t last_site;            // site code read by the last failing spv_check
+  struct SpvProf* prof;          // event record of spv_profile_enable (NULL until first enabled)
+  int32_t prof_on;
+};
+
+// Event pair around one launch group while profiling is on (no-ops otherwise).
+int32_t spv_prof_begin(spv_ctx* ctx, int32_t cls, cudaStream_t stream);
+void spv_prof_end(spv_ctx* ctx, int32_t token, cudaStream_t stream, double work);
+struct SpvProfScope {
+  spv_ctx* ctx; cudaStream_t stream; int32_t token; double work;
+  SpvProfScope(spv_ctx* c, int32_t cls, cudaStream_t s, double w = 0.0)
+      : ctx(c), stream(s), token(c->prof_on ? spv_prof_begin(c, cls, s) : -1), work(w) {}
+  ~SpvProfScope() { if (token >= 0) spv_prof_end(ctx, token, stream, work); }
 };
 
 #define SPV_CUDA_OK(expr)                         \

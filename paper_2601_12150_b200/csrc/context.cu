@@ -2,6 +2,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <vector>
+
 #include "common.cuh"
 
 extern "C" int32_t spv_create(spv_ctx** out, int32_t device) {
@@ -32,9 +34,68 @@ extern "C" int32_t spv_create(spv_ctx** out, int32_t device) {
   return SPV_OK;
 }
 
+// ---- per-class event timing ------------------------------------------------------------------
+struct SpvProfRec { cudaEvent_t e0, e1; int32_t cls; double work; };
+struct SpvProf {
+  std::vector<SpvProfRec> recs;        // event pairs, reused after every read
+  size_t used = 0;
+};
+
+int32_t spv_prof_begin(spv_ctx* ctx, int32_t cls, cudaStream_t stream) {
+  SpvProf* p = ctx->prof;
+  if (!p) return -1;
+  if (p->used == p->recs.size()) {
+    SpvProfRec r{};
+    if (cudaEventCreate(&r.e0) != cudaSuccess || cudaEventCreate(&r.e1) != cudaSuccess) return -1;
+    p->recs.push_back(r);
+  }
+  SpvProfRec& r = p->recs[p->used];
+  r.cls = cls;
+  r.work = 0.0;
+  if (cudaEventRecord(r.e0, stream) != cudaSuccess) return -1;
+  return (int32_t)p->used++;
+}
+
+void spv_prof_end(spv_ctx* ctx, int32_t token, cudaStream_t stream, double work) {
+  SpvProfRec& r = ctx->prof->recs[(size_t)token];
+  r.work = work;
+  cudaEventRecord(r.e1, stream);
+}
+
+extern "C" int32_t spv_profile_enable(spv_ctx* ctx, int32_t enable) {
+  if (!ctx) return SPV_ERR_INVALID_ARG;
+  if (enable && !ctx->prof) ctx->prof = new SpvProf();
+  if (ctx->prof) ctx->prof->used = 0;
+  ctx->prof_on = enable ? 1 : 0;
+  return SPV_OK;
+}
+
+extern "C" int32_t spv_profile_read(spv_ctx* ctx, spv_kernel_stat* out) {
+  if (!ctx || !out) return SPV_ERR_INVALID_ARG;
+  SpvProf* p = ctx->prof;
+  if (!p) return SPV_OK;
+  for (size_t i = 0; i < p->used; ++i) {
+    SpvProfRec& r = p->recs[i];
+    SPV_CUDA_OK(cudaEventSynchronize(r.e1));
+    float ms = 0.f;
+    SPV_CUDA_OK(cudaEventElapsedTime(&ms, r.e0, r.e1));
+    if (r.cls >= 0 && r.cls < SPV_K_COUNT) {
+      out[r.cls].launches += 1;
+      out[r.cls].ms += (double)ms;
+      out[r.cls].work += r.work;
+    }
+  }
+  p->used = 0;
+  return SPV_OK;
+}
+
 extern "C" int32_t spv_destroy(spv_ctx* ctx) {
   if (!ctx) return SPV_ERR_INVALID_ARG;
   cudaSetDevice(ctx->device);
+  if (ctx->prof) {
+    for (SpvProfRec& r : ctx->prof->recs) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+    delete ctx->prof;
+  }
   cudaFree(ctx->d_status);
   free(ctx);
   return SPV_OK;

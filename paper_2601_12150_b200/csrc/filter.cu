@@ -240,9 +240,13 @@ extern "C" int32_t cls_score_topk_filter(spv_ctx* ctx, const spv_filter_desc* d,
   uint32_t* key_ws =
       (uint32_t*)((char*)workspace + spv_align_up((size_t)d->batch * npad * sizeof(float), 256));
 
-  filter_mean_key<<<dim3((npad + 255) / 256, d->batch), 256, 0, stream>>>(scores, d->heads, d->n_patch, npad,
-                                                                        mean_ws, key_ws, mean_scores);
-  filter_select<<<d->batch, kSelThreads, 0, stream>>>(key_ws, d->n_patch, npad, k, kept_idx, pos_in, pos_out);
+  {
+    SpvProfScope prof(ctx, SPV_K_FILTER_SELECT, stream,
+                      (double)d->batch * ((double)d->heads * d->n_patch * 4.0 + (double)k * 4.0));
+    filter_mean_key<<<dim3((npad + 255) / 256, d->batch), 256, 0, stream>>>(scores, d->heads, d->n_patch, npad,
+                                                                          mean_ws, key_ws, mean_scores);
+    filter_select<<<d->batch, kSelThreads, 0, stream>>>(key_ws, d->n_patch, npad, k, kept_idx, pos_in, pos_out);
+  }
   int launches = 2;
   if (tokens_in) {
     const int64_t rows = (int64_t)d->batch * (d->n_global + k);
@@ -252,6 +256,7 @@ extern "C" int32_t cls_score_topk_filter(spv_ctx* ctx, const spv_filter_desc* d,
     int64_t blocks = (rows + 7) / 8;
     const int64_t cap = (int64_t)ctx->sm_count * 8;
     if (blocks > cap) blocks = cap;
+    SpvProfScope prof(ctx, SPV_K_FILTER_GATHER, stream, 2.0 * (double)rows * d->dim * 2.0);
     filter_gather<<<(unsigned)blocks, 256, 0, stream>>>((const uint4*)tokens_in, (uint4*)tokens_out, kept_idx,
                                                        d->batch, d->n_global, k, row_vec, in_sb / 8, out_sb / 8);
     ++launches;

@@ -213,6 +213,7 @@ int32_t launch(spv_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tw, const
   }
   const int tiles = ((d->m + BM - 1) / BM) * ((d->n + BN - 1) / BN);
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  SpvProfScope prof(ctx, SPV_K_GEMM, stream, 2.0 * (double)d->m * (double)d->n * (double)d->k);
   gemm_bf16_kernel<EPI><<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tw, d->m, d->n, d->k, ep, ctx->d_status);
   return spv_launch_ok(ctx);
 }

@@ -90,6 +90,7 @@ extern "C" int32_t spv_layernorm(spv_ctx* ctx, const float* x, int64_t rows, int
   int64_t blocks = (rows + 7) / 8;
   const int64_t cap = (int64_t)ctx->sm_count * 8;
   if (blocks > cap) blocks = cap;
+  SpvProfScope prof(ctx, SPV_K_LAYERNORM, (cudaStream_t)stream, (double)rows * dim * 6.0);
   layernorm_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(x, rows, dim, gamma, beta, eps,
                                                                       (__nv_bfloat16*)y, out_row);
   return spv_launch_ok(ctx);

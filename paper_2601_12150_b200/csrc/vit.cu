@@ -283,6 +283,7 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
   int32_t* out_row = (int32_t*)(ws + L.out_row);
 
   // ---- token order tables, patch embedding (a1)
+  SpvProfScope* prof_misc = new SpvProfScope(ctx, SPV_K_MISC, stream);
   vit_bm_tables<<<cdiv(np0, 256), 256, 0, stream>>>(gh, gw, c->block, L.nbx, bm_pos, bm_of_pos, batch);
   vit_permute_pos<<<cdiv((int64_t)np0 * (D / 4), 256), 256, 0, stream>>>((const float4*)w->pos, bm_pos, G, np0,
                                                                           D / 4, (float4*)pos_bm);
@@ -299,6 +300,7 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
     w_pe = w_pe_pad;
     launches += 2;
   }
+  delete prof_misc;
   if ((st = spv_launch_ok(ctx, launches)) != SPV_OK) return st;
   for (int b = 0; b < batch; ++b) {
     spv_gemm_desc g{};
@@ -391,9 +393,12 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
       }
       // the kept set as a one-head score row over the internal order; ranking it compacts the
       // residual stream (fp32 rows copied as 2*D 16-bit elements) and the positions, order kept
-      SPV_CUDA_OK(cudaMemsetAsync(mark, 0, (size_t)batch * np0 * 4, stream));
-      vit_mark_kept<<<dim3(cdiv(k, 256), batch), 256, 0, stream>>>(kept_positions, k, np0, mark);
-      vit_mask_to_order<<<dim3(cdiv(np0, 256), batch), 256, 0, stream>>>(mark, bm_pos, np0, mask);
+      {
+        SpvProfScope prof(ctx, SPV_K_MISC, stream);
+        SPV_CUDA_OK(cudaMemsetAsync(mark, 0, (size_t)batch * np0 * 4, stream));
+        vit_mark_kept<<<dim3(cdiv(k, 256), batch), 256, 0, stream>>>(kept_positions, k, np0, mark);
+        vit_mask_to_order<<<dim3(cdiv(np0, 256), batch), 256, 0, stream>>>(mark, bm_pos, np0, mask);
+      }
       if ((st = spv_launch_ok(ctx, 2)) != SPV_OK) return st;
       spv_filter_desc fd{};
       fd.batch = batch; fd.heads = 1; fd.n_patch = np0; fd.n_global = G; fd.dim = 2 * D; fd.keep_ratio = c->keep_ratio;
@@ -414,10 +419,13 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
   }
 
   // ---- final LayerNorm, rows scattered back to ascending original position (a12)
-  if (c->filter_layer > 0) {
-    vit_out_rows_kept<<<batch, 1024, 0, stream>>>(mark, np0, pos2, L.k, G, rank, out_row);
-  } else {
-    vit_out_rows_full<<<dim3(cdiv(L.n0, 256), batch), 256, 0, stream>>>(bm_pos, G, np0, out_row);
+  {
+    SpvProfScope prof(ctx, SPV_K_MISC, stream);
+    if (c->filter_layer > 0) {
+      vit_out_rows_kept<<<batch, 1024, 0, stream>>>(mark, np0, pos2, L.k, G, rank, out_row);
+    } else {
+      vit_out_rows_full<<<dim3(cdiv(L.n0, 256), batch), 256, 0, stream>>>(bm_pos, G, np0, out_row);
+    }
   }
   if ((st = spv_launch_ok(ctx)) != SPV_OK) return st;
   return spv_layernorm(ctx, x, (int64_t)batch * n, D, w->lnf_g, w->lnf_b, c->ln_eps, out_tokens, out_row, stream);
