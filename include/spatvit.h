@@ -41,7 +41,8 @@ enum {
   SPV_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or smaller than the query says */
   SPV_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed                          */
   SPV_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (reported by spv_check)   */
-  SPV_ERR_ALIGNMENT = 6    /* a tensor base or stride breaks the 16-byte rule              */
+  SPV_ERR_ALIGNMENT = 6,   /* a tensor base or stride breaks the 16-byte rule              */
+  SPV_ERR_STATIC_LIMIT = 7 /* request larger than the library's built-in scratch array     */
 };
 
 typedef struct spv_ctx spv_ctx; /* device id, device status word, cached driver entry points */
@@ -131,6 +132,37 @@ int32_t cls_score_topk_filter(spv_ctx* ctx, const spv_filter_desc* desc, const f
                               const void* tokens_in, void* tokens_out, int32_t* kept_idx,
                               float* mean_scores, const int32_t* pos_in, int32_t* pos_out,
                               void* workspace, size_t workspace_bytes, void* stream);
+
+/* The token filter for callers that must not allocate device memory (the paper has no
+ * counterpart; this is a packaging variant of cls_score_topk_filter, same kernels, same results).
+ *
+ * Who needs it: code that runs after an application has handed out all of its device memory
+ * and forbids further allocation (an inference server with a fixed memory plan, a plug-in
+ * inside a host program that owns the allocator), and code in a latency-critical loop where
+ * cudaMalloc / cudaFree would synchronise the whole device.  Such callers can neither size a
+ * workspace and allocate it nor create an spv_ctx (spv_create allocates), so this entry point
+ * takes no context and no workspace: the head means and ranking keys live in a file-scope
+ * device array of SPV_FILTER_STATIC_BYTES that every GPU holds from the moment the library is
+ * loaded until the process exits.
+ *
+ * Limits and rules
+ *   - batch * round_up(n_patch, 4) * 8 bytes must fit in SPV_FILTER_STATIC_BYTES (2 MiB: e.g.
+ *     4 images of a 256 x 256 patch grid); larger requests return SPV_ERR_STATIC_LIMIT and
+ *     launch nothing;
+ *   - works on the CUDA device that is current on the calling thread.  The first call on a
+ *     device looks up the array's device address (one cudaGetSymbolAddress, no allocation) and
+ *     keeps it; make that first call before any stream capture begins;
+ *   - all calls on one device share the array, and it keeps what the previous call left there.
+ *     The kernels write every element they later read, so no clearing is needed, but two calls
+ *     whose kernels can overlap on the GPU (different streams without an ordering) race on it:
+ *     order them;
+ *   - the call itself performs no cudaMalloc, cudaFree or other allocating routine; inputs and
+ *     outputs are the caller's, exactly as for cls_score_topk_filter.  Asynchronous on `stream`. */
+#define SPV_FILTER_STATIC_BYTES (2u << 20)
+int32_t cls_score_topk_filter_static(const spv_filter_desc* desc, const float* scores,
+                                     const void* tokens_in, void* tokens_out, int32_t* kept_idx,
+                                     float* mean_scores, const int32_t* pos_in, int32_t* pos_out,
+                                     void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * Sec. 3 / Sec. 4.1 -- the ViT backbone run with sparse attention and the filter.

@@ -11,7 +11,8 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libspatvit.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_ALIGNMENT = range(7)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_ALIGNMENT, ERR_STATIC_LIMIT = range(8)
+FILTER_STATIC_BYTES = 2 << 20
 TOKENS_ROW_MAJOR, TOKENS_BLOCK_MAJOR = 0, 1
 MLP_GELU, MLP_SWIGLU = 0, 1
 ATTN_DENSE, ATTN_SPARSE = 0, 1
@@ -20,6 +21,7 @@ EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_SILU, EPI_BIAS_MUL, EPI_BIAS_SCALE_RESID, EPI_
 EXPORTS = ["spv_create", "spv_destroy", "spv_status_string", "spv_check", "spv_last_wait_site", "spv_launch_count",
            "spv_attn_workspace_size", "spatial_block_attention",
            "spv_filter_keep_count", "spv_filter_workspace_size", "cls_score_topk_filter",
+           "cls_score_topk_filter_static",
            "spv_vit_workspace_size", "vit_forward", "spv_gemm_bf16", "spv_layernorm",
            "spv_profile_enable", "spv_profile_read"]
 
@@ -106,6 +108,7 @@ def lib():
         L.spv_filter_workspace_size.argtypes = [C.POINTER(FilterDesc), C.POINTER(C.c_size_t)]
         L.cls_score_topk_filter.argtypes = [C.c_void_p, C.POINTER(FilterDesc)] + [C.c_void_p] * 8 + \
             [C.c_size_t, C.c_void_p]
+        L.cls_score_topk_filter_static.argtypes = [C.POINTER(FilterDesc)] + [C.c_void_p] * 8
         L.spv_attn_workspace_size.argtypes = [C.POINTER(AttnDesc), C.POINTER(C.c_size_t)]
         L.spatial_block_attention.argtypes = [C.c_void_p, C.POINTER(AttnDesc)] + [C.c_void_p] * 6 + \
             [C.c_size_t, C.c_void_p]
@@ -147,6 +150,25 @@ def filter_keep_count(n_patch, keep_ratio):
     k = C.c_int32(0)
     _raise(lib().spv_filter_keep_count(int(n_patch), float(keep_ratio), C.byref(k)), "spv_filter_keep_count")
     return k.value
+
+
+def cls_score_topk_filter_static(scores, tokens_in, tokens_out, kept_idx, n_global=1, keep_ratio=0.5,
+                                 mean_scores=None, pos_in=None, pos_out=None, stream=None):
+    """The token filter through the entry point that allocates nothing: no context, no workspace
+    (its scratch is a 2 MiB array built into the library), and this wrapper creates no tensor
+    either -- every output is the caller's.  For callers that run under a fixed device-memory
+    plan or inside a loop where an allocation would stall the device.  Works on the current CUDA
+    device; calls that may overlap on the GPU must be ordered by the caller (shared scratch).
+    scores fp32 [B, h, n_patch]; tokens_in / tokens_out bf16 [B, G+n_patch, dim] / [B, G+k, dim] or
+    both None; kept_idx int32 [B, k]."""
+    B, H, NP = scores.shape
+    dim = 0 if tokens_in is None else tokens_in.shape[-1]
+    d = FilterDesc(B, H, NP, n_global, dim, float(keep_ratio), 0, 0)
+    st = lib().cls_score_topk_filter_static(C.byref(d), _ptr(scores), _ptr(tokens_in), _ptr(tokens_out),
+                                            _ptr(kept_idx), _ptr(mean_scores), _ptr(pos_in), _ptr(pos_out),
+                                            _stream(stream))
+    _raise(st, "cls_score_topk_filter_static")
+    return tokens_out, kept_idx
 
 
 class Context:

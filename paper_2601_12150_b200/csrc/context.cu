@@ -110,6 +110,7 @@ extern "C" const char* spv_status_string(int32_t s) {
     case SPV_ERR_CUDA: return "CUDA call failed";
     case SPV_ERR_TIMEOUT: return "bounded device-side wait expired";
     case SPV_ERR_ALIGNMENT: return "tensor base or stride not 16-byte aligned";
+    case SPV_ERR_STATIC_LIMIT: return "request exceeds the built-in static scratch array";
     default: return "unknown status";
   }
 }

@@ -263,3 +263,79 @@ extern "C" int32_t cls_score_topk_filter(spv_ctx* ctx, const spv_filter_desc* d,
   }
   return spv_launch_ok(ctx, launches);
 }
+
+// ------------------------------------------------------------------------------------------
+// Variant for callers that cannot allocate: the scratch (head means + ranking keys) is a
+// file-scope device array instead of a caller workspace.  In host code `g_filter_scratch` is only
+// a stand-in for the symbol, not a device address: the address is looked up once per device with
+// cudaGetSymbolAddress and that pointer is what the kernels receive.
+// ------------------------------------------------------------------------------------------
+#include <mutex>
+
+static __device__ __align__(256) unsigned char g_filter_scratch[SPV_FILTER_STATIC_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices];     // device address of g_filter_scratch on each device
+int g_static_sms[kMaxDevices];
+
+// Set-up of the current device (first call only): symbol address and SM count.  No allocation.
+int32_t static_scratch(int* device_out, void** ptr_out, int* sms_out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPV_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_filter_scratch) != cudaSuccess || !p) return SPV_ERR_CUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+      return SPV_ERR_CUDA;
+    g_static_sms[dev] = sms;
+    g_static_ptr[dev] = p;
+  }
+  *device_out = dev;
+  *ptr_out = g_static_ptr[dev];
+  *sms_out = g_static_sms[dev];
+  return SPV_OK;
+}
+}  // namespace
+
+extern "C" int32_t cls_score_topk_filter_static(const spv_filter_desc* d, const float* scores, const void* tokens_in,
+                                                void* tokens_out, int32_t* kept_idx, float* mean_scores,
+                                                const int32_t* pos_in, int32_t* pos_out, void* stream_) {
+  int32_t k;
+  int32_t st = validate(d, &k);
+  if (st != SPV_OK) return st;
+  if (!scores || !kept_idx) return SPV_ERR_INVALID_ARG;
+  if ((tokens_in == nullptr) != (tokens_out == nullptr)) return SPV_ERR_INVALID_ARG;
+  if (tokens_in && d->dim == 0) return SPV_ERR_INVALID_ARG;
+  if (((uintptr_t)scores & 15u) || ((uintptr_t)tokens_in & 15u) || ((uintptr_t)tokens_out & 15u))
+    return SPV_ERR_ALIGNMENT;
+  const size_t npad = spv_align_up((size_t)d->n_patch, 4);
+  const size_t half = spv_align_up((size_t)d->batch * npad * sizeof(float), 256);
+  if (2 * half > (size_t)SPV_FILTER_STATIC_BYTES) return SPV_ERR_STATIC_LIMIT;
+  int dev, sms;
+  void* scratch;
+  if ((st = static_scratch(&dev, &scratch, &sms)) != SPV_OK) return st;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  float* mean_ws = (float*)scratch;
+  uint32_t* key_ws = (uint32_t*)((char*)scratch + half);
+  // every element of [0, npad) per image is written by filter_mean_key before filter_select reads
+  // it, so what an earlier call left in the array is never seen
+  filter_mean_key<<<dim3((unsigned)((npad + 255) / 256), d->batch), 256, 0, stream>>>(
+      scores, d->heads, d->n_patch, (int)npad, mean_ws, key_ws, mean_scores);
+  filter_select<<<d->batch, kSelThreads, 0, stream>>>(key_ws, d->n_patch, (int)npad, k, kept_idx, pos_in, pos_out);
+  if (tokens_in) {
+    const int64_t rows = (int64_t)d->batch * (d->n_global + k);
+    const int row_vec = d->dim / 8;
+    const int64_t in_sb = d->in_stride_b ? d->in_stride_b : (int64_t)(d->n_global + d->n_patch) * d->dim;
+    const int64_t out_sb = d->out_stride_b ? d->out_stride_b : (int64_t)(d->n_global + k) * d->dim;
+    int64_t blocks = (rows + 7) / 8;
+    const int64_t cap = (int64_t)sms * 8;
+    if (blocks > cap) blocks = cap;
+    filter_gather<<<(unsigned)blocks, 256, 0, stream>>>((const uint4*)tokens_in, (uint4*)tokens_out, kept_idx,
+                                                       d->batch, d->n_global, k, row_vec, in_sb / 8, out_sb / 8);
+  }
+  return cudaGetLastError() == cudaSuccess ? SPV_OK : SPV_ERR_CUDA;
+}
