@@ -27,7 +27,8 @@ constexpr int TQ = 128;            // query rows per tile (MMA M)
 constexpr int TK = 128;            // keys per tile (MMA N of S, K extent of P V)
 constexpr int HD = 64;             // head_dim
 constexpr int KST = 2;             // K / V smem stages
-constexpr int ATT_THREADS = 192;   // warps 0-3 softmax, 4 TMA, 5 MMA
+constexpr int ATT_THREADS = 256;   // warps 0-3 softmax (one warpgroup), 4 TMA, 5 MMA, 6-7 idle: the second
+                                   // warpgroup exists so that it can hand its registers to the first
 constexpr int TILE_BYTES = 128 * 128;
 constexpr int ATT_SMEM = TILE_BYTES * (1 + 2 * KST) + 1024 + 256;
 constexpr int MAXG = 8;
@@ -276,6 +277,10 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // the softmax warpgroup holds a whole 128-column score row per thread; the other warpgroup
+  // needs few registers
+  if (warp >= 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 32;");
   if (warp == 4) {
     // ---------------- TMA producer
     if (lane == 0) {
@@ -336,7 +341,9 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tc_commit(&v_empty[s]);
       }
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
     // ---------------- softmax + epilogue: thread `row` owns query row `row` (TMEM lane `row`)
     const int row = threadIdx.x;
     const int tok = q_begin + row;
@@ -384,32 +391,51 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     for (int cy = cy0; cy <= cy1; ++cy) {
       const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
       int lo = __ldg(boff + cy * p.nbx + rlo), hi = __ldg(boff + cy * p.nbx + rhi + 1);
-      if (!valid) hi = lo;
+      // Rows past the end of the tile are never stored: they take the key range of the warp's
+      // first row, so that the warp stays uniform (valid rows are a prefix of the tile).
+      {
+        const int lo0 = __shfl_sync(0xffffffffu, lo, 0), hi0 = __shfl_sync(0xffffffffu, hi, 0);
+        const bool v0 = __shfl_sync(0xffffffffu, (int)valid, 0) != 0;
+        if (!valid) { lo = lo0; hi = v0 ? hi0 : lo0; }
+      }
       for (int kb = ks; kb < ke; kb += TK, ++j) {
-        // this row's allowed keys are the tile columns [c_lo, c_hi)
+        // this row's allowed keys are the tile columns [c_lo, c_hi); u_* is the union over the
+        // warp's rows (columns outside it are not even read), i_* the intersection (columns
+        // inside it need no per-element mask)
         const int c_lo = min(max(lo - kb, 0), TK), c_hi = min(max(hi - kb, 0), TK);
         const bool some = c_lo < c_hi;
-        int w_lo = some ? c_lo : TK, w_hi = some ? c_hi : 0;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          w_lo = min(w_lo, __shfl_xor_sync(0xffffffffu, w_lo, o));
-          w_hi = max(w_hi, __shfl_xor_sync(0xffffffffu, w_hi, o));
-        }
+        const int u_lo = __reduce_min_sync(0xffffffffu, some ? c_lo : TK);
+        const int u_hi = __reduce_max_sync(0xffffffffu, some ? c_hi : 0);
+        const int i_lo = __reduce_max_sync(0xffffffffu, some ? c_lo : TK);
+        const int i_hi = __reduce_min_sync(0xffffffffu, some ? c_hi : 0);
         mbar_wait(s_full, j & 1, abort_flag, p.status, 0x1800);
         tc_fence_after();
-        // pass 1: row maximum over the allowed columns
+        // one pass: the live 32-column chunks of S go to registers, then S is released
+        uint32_t sr[TK];
+#pragma unroll
+        for (int c = 0; c < TK / 32; ++c)
+          if (32 * c < u_hi && 32 * c + 32 > u_lo) tmem_ld32(lane_addr + S_COL + 32 * c, sr + 32 * c);
+        tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(s_free);                               // S may be overwritten by the next Q K^T
         float mx = -INFINITY;
 #pragma unroll
         for (int c = 0; c < TK / 32; ++c) {
-          if (32 * c < w_hi && 32 * c + 32 > w_lo) {
-            uint32_t sr[32];
-            tmem_ld32(lane_addr + S_COL + 32 * c, sr);
-            tc_wait_ld();
+          if (32 * c < u_hi && 32 * c + 32 > u_lo) {
+            if (!(32 * c >= i_lo && 32 * c + 32 <= i_hi)) {   // boundary chunk: mask per element
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int col = 32 * c + i;
-              if (col >= c_lo && col < c_hi) mx = fmaxf(mx, __uint_as_float(sr[i]));
+              for (int i = 0; i < 32; ++i)
+                if (32 * c + i < c_lo || 32 * c + i >= c_hi) sr[32 * c + i] = 0xff800000u;
             }
+            float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              m0 = fmaxf(m0, __uint_as_float(sr[32 * c + i]));
+              m1 = fmaxf(m1, __uint_as_float(sr[32 * c + i + 1]));
+              m2 = fmaxf(m2, __uint_as_float(sr[32 * c + i + 2]));
+              m3 = fmaxf(m3, __uint_as_float(sr[32 * c + i + 3]));
+            }
+            mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
           }
         }
         // lazy rescale: the running maximum only moves when it would grow by more than 2^8
@@ -418,34 +444,6 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const float m_new = need ? m_t : m;
         const float alpha = need ? fast_exp2(m - m_new) : 1.0f;
         const bool any_need = __any_sync(0xffffffffu, need);
-        // pass 2: p = 2^(s*scale - m), packed to bf16 pairs
-        uint32_t pk[TK / 2];
-        float rowsum = 0.f;
-#pragma unroll
-        for (int c = 0; c < TK / 32; ++c) {
-          if (32 * c < w_hi && 32 * c + 32 > w_lo) {
-            uint32_t sr[32];
-            tmem_ld32(lane_addr + S_COL + 32 * c, sr);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const int col = 32 * c + i;
-              float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), sl2, -m_new));
-              float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), sl2, -m_new));
-              if (!(col >= c_lo && col < c_hi)) p0 = 0.f;
-              if (!(col + 1 >= c_lo && col + 1 < c_hi)) p1 = 0.f;
-              rowsum += p0 + p1;
-              pk[16 * c + i / 2] = pack_bf16(p0, p1);
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) pk[16 * c + i] = 0u;
-          }
-        }
-        l = l * alpha + rowsum;
-        m = m_new;
-        tc_fence_before();
-        mbar_arrive(s_free);                               // S may be overwritten by the next Q K^T
         if (j > 0) {
           mbar_wait(pv_done, (j - 1) & 1, abort_flag, p.status, 0x1900);   // P buffer and O are free
           tc_fence_after();
@@ -461,8 +459,29 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
           }
         }
+        // p = 2^(s*scale - m) chunk by chunk, packed to bf16 pairs and written to TMEM at once
+        // (masked scores are -inf, so p = 0)
+        float rs0 = 0.f, rs1 = 0.f;
 #pragma unroll
-        for (int c = 0; c < TK / 32; ++c) tmem_st16(lane_addr + P_COL + 16 * c, pk + 16 * c);
+        for (int c = 0; c < TK / 32; ++c) {
+          uint32_t pk[16];
+          if (32 * c < u_hi && 32 * c + 32 > u_lo) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              const float p0 = fast_exp2(fmaf(__uint_as_float(sr[32 * c + i]), sl2, -m_new));
+              const float p1 = fast_exp2(fmaf(__uint_as_float(sr[32 * c + i + 1]), sl2, -m_new));
+              rs0 += p0;
+              rs1 += p1;
+              pk[i / 2] = pack_bf16(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+          }
+          tmem_st16(lane_addr + P_COL + 16 * c, pk);
+        }
+        l = l * alpha + (rs0 + rs1);
+        m = m_new;
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(p_full);

@@ -117,17 +117,29 @@ __device__ __forceinline__ uint64_t global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-static __device__ __noinline__ void mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                            uint32_t* status, uint32_t site) {
+// try_wait that lets the hardware park the thread for up to `ns` nanoseconds (it wakes as soon as
+// the phase completes): a waiting warp then takes no issue slots from the working warps of its SM
+// sub-partition, which a hot polling loop does.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+static __device__ __forceinline__ void mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                      uint32_t* status, uint32_t site) {
   const uint64_t t0 = global_ns();
-  for (uint32_t it = 0;; ++it) {
-    if (mbar_try_wait(bar, parity)) return;
-    if ((it & 63u) == 63u) {
-      if (*abort_flag) return;
-      // another CTA already gave up: do not wait out a second limit here
-      if (*reinterpret_cast<volatile uint32_t*>(status) != 0u) { *abort_flag = 1; return; }
-      if (global_ns() - t0 > SPV_WAIT_LIMIT_NS) break;
-    }
+  for (;;) {
+    if (mbar_try_wait_parked(bar, parity, 20000u)) return;
+    if (*abort_flag) return;
+    // another CTA already gave up: do not wait out a second limit here
+    if (*reinterpret_cast<volatile uint32_t*>(status) != 0u) { *abort_flag = 1; return; }
+    if (global_ns() - t0 > SPV_WAIT_LIMIT_NS) break;
   }
   *abort_flag = 1;
   atomicCAS(status, 0u, site);
