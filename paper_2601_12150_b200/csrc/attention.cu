@@ -30,7 +30,9 @@ constexpr int KST = 2;             // K / V smem stages
 constexpr int ATT_THREADS = 256;   // warps 0-3 softmax (one warpgroup), 4 TMA, 5 MMA, 6-7 idle: the second
                                    // warpgroup exists so that it can hand its registers to the first
 constexpr int TILE_BYTES = 128 * 128;
-constexpr int ATT_SMEM = TILE_BYTES * (1 + 2 * KST) + 1024 + 256;
+constexpr int GROW_BYTES = 1024;   // global-token rows of one head: up to 8 x 128 B
+constexpr int ATT_SMEM = TILE_BYTES * (1 + 2 * KST) + 2 * GROW_BYTES + 1024 /*align*/ + 256 /*barriers*/ +
+                         8 * 128 * 4 /*global-token scores*/;
 constexpr int MAXG = 8;
 constexpr uint32_t TMEM_COLS = 256;
 constexpr uint32_t S_COL = 0, P_COL = 128, O_COL = 192;
@@ -224,7 +226,8 @@ __device__ __forceinline__ void unpack8(const uint4& u, float* f) {
 
 __global__ void __launch_bounds__(ATT_THREADS, 2)
 attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                  const __grid_constant__ CUtensorMap tm_v, const PatchParams p) {
+                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kg,
+                  const __grid_constant__ CUtensorMap tm_vg, const PatchParams p) {
   const int b = blockIdx.z, h = blockIdx.y;
   const int4 tile = __ldg(p.tiles + (size_t)b * p.tiles_per_image + blockIdx.x);
   const int q_begin = tile.x, q_end = tile.y;
@@ -236,7 +239,9 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   uint8_t* sQ = smem;
   uint8_t* sK = smem + TILE_BYTES;
   uint8_t* sV = smem + TILE_BYTES * (1 + KST);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + TILE_BYTES * (1 + 2 * KST));
+  uint8_t* sKg = smem + TILE_BYTES * (1 + 2 * KST);      // global-token key rows (G x 128 B, swizzled)
+  uint8_t* sVg = sKg + GROW_BYTES;                       // global-token value rows
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sVg + GROW_BYTES);
   uint64_t* q_full = bars;
   uint64_t* k_full = bars + 1;
   uint64_t* k_empty = k_full + KST;
@@ -248,6 +253,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   uint64_t* pv_done = p_full + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + 1);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* s_sg = reinterpret_cast<float*>(bars + 32);     // [G][128] scaled scores of the global keys
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = p.radius, G = p.n_global;
@@ -285,8 +291,10 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // ---------------- TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
-      mbar_expect_tx(q_full, TILE_BYTES);
+      mbar_expect_tx(q_full, TILE_BYTES + 2 * G * 128);
       tma_load_4d(sQ, &tm_q, q_full, 0, G + q_begin, h, b);
+      tma_load_4d(sKg, &tm_kg, q_full, 0, 0, h, b);
+      tma_load_4d(sVg, &tm_vg, q_full, 0, 0, h, b);
       uint32_t j = 0;
       for (int cy = cy0; cy <= cy1; ++cy) {
         const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
@@ -356,7 +364,6 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     // global tokens: initial softmax state (m, l); their value rows are added in the epilogue
     mbar_wait(q_full, 0, abort_flag, p.status, 0x1700);
-    float sg[MAXG];
     float m = -INFINITY;
     {
       float qf[HD];
@@ -365,27 +372,27 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const uint4 u = *reinterpret_cast<const uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4));
         unpack8(u, qf + 8 * c);
       }
+#pragma unroll 1
+      for (int g = 0; g < G; ++g) {
+        float d0 = 0.f, d1 = 0.f;
 #pragma unroll
-      for (int g = 0; g < MAXG; ++g) {
-        sg[g] = -INFINITY;
-        if (g < G) {
-          const uint4* kg = reinterpret_cast<const uint4*>(p.k + b * p.sb + (int64_t)g * p.st + (int64_t)h * p.sh);
-          float dot = 0.f;
+        for (int c = 0; c < 8; ++c) {
+          float kf[8];
+          unpack8(*reinterpret_cast<const uint4*>(sKg + g * 128 + ((c ^ (g & 7)) << 4)), kf);
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            float kf[8];
-            unpack8(__ldg(kg + c), kf);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) dot = fmaf(qf[8 * c + i], kf[i], dot);
+          for (int i = 0; i < 8; i += 2) {
+            d0 = fmaf(qf[8 * c + i], kf[i], d0);
+            d1 = fmaf(qf[8 * c + i + 1], kf[i + 1], d1);
           }
-          sg[g] = dot * sl2;
-          m = fmaxf(m, sg[g]);
         }
+        const float sc = (d0 + d1) * sl2;
+        s_sg[g * 128 + row] = sc;
+        m = fmaxf(m, sc);
       }
     }
     float l = 0.f;
-#pragma unroll
-    for (int g = 0; g < MAXG; ++g) if (g < G) l += fast_exp2(sg[g] - m);
+#pragma unroll 1
+    for (int g = 0; g < G; ++g) l += fast_exp2(s_sg[g * 128 + row] - m);
 
     uint32_t j = 0;
     for (int cy = cy0; cy <= cy1; ++cy) {
@@ -410,6 +417,21 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const int i_hi = __reduce_min_sync(0xffffffffu, some ? c_hi : 0);
         mbar_wait(s_full, j & 1, abort_flag, p.status, 0x1800);
         tc_fence_after();
+        // boundary chunks (some of the warp's rows see only part of them) are masked in place
+        // first, by a small loop, so that the unrolled main pass below carries no mask code
+#pragma unroll 1
+        for (int cb = 0; cb < TK; cb += 32) {
+          if (cb < u_hi && cb + 32 > u_lo && !(cb >= i_lo && cb + 32 <= i_hi)) {
+            uint32_t t[32];
+            tmem_ld32(lane_addr + S_COL + cb, t);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (cb + i < c_lo || cb + i >= c_hi) t[i] = 0xff800000u;
+            tmem_st32(lane_addr + S_COL + cb, t);
+          }
+        }
+        tc_wait_st();
         // one pass: the live 32-column chunks of S go to registers, then S is released
         uint32_t sr[TK];
 #pragma unroll
@@ -422,11 +444,6 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
         for (int c = 0; c < TK / 32; ++c) {
           if (32 * c < u_hi && 32 * c + 32 > u_lo) {
-            if (!(32 * c >= i_lo && 32 * c + 32 <= i_hi)) {   // boundary chunk: mask per element
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (32 * c + i < c_lo || 32 * c + i >= c_hi) sr[32 * c + i] = 0xff800000u;
-            }
             float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
@@ -506,24 +523,21 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
       for (int i = 0; i < 32; ++i) of[32 * c + i] = __uint_as_float(orr[i]);
     }
+#pragma unroll 1
+    for (int g = 0; g < G; ++g) {
+      const float w = fast_exp2(s_sg[g * 128 + row] - m);
 #pragma unroll
-    for (int g = 0; g < MAXG; ++g) {
-      if (g < G) {
-        const float w = fast_exp2(sg[g] - m);
-        const uint4* vg = reinterpret_cast<const uint4*>(p.v + b * p.sb + (int64_t)g * p.st + (int64_t)h * p.sh);
+      for (int c = 0; c < 8; ++c) {
+        float vf[8];
+        unpack8(*reinterpret_cast<const uint4*>(sVg + g * 128 + ((c ^ (g & 7)) << 4)), vf);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          float vf[8];
-          unpack8(__ldg(vg + c), vf);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) of[8 * c + i] = fmaf(w, vf[i], of[8 * c + i]);
-        }
+        for (int i = 0; i < 8; ++i) of[8 * c + i] = fmaf(w, vf[i], of[8 * c + i]);
       }
     }
-    if (valid) {
+    // stage the bf16 row in the (now dead) Q tile, same 128-byte swizzle; each warp then stores its
+    // own 32 rows, eight lanes per 128-byte row
+    {
       const float inv = 1.0f / l;
-      const int ot = p.o_tok ? __ldg(p.o_tok + (size_t)b * p.n_patch + tok) : tok;
-      uint4* dst = reinterpret_cast<uint4*>(p.o + b * p.o_sb + (int64_t)(G + ot) * p.o_st + (int64_t)h * p.o_sh);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         uint4 w;
@@ -531,7 +545,18 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         w.y = pack_bf16(of[8 * c + 2] * inv, of[8 * c + 3] * inv);
         w.z = pack_bf16(of[8 * c + 4] * inv, of[8 * c + 5] * inv);
         w.w = pack_bf16(of[8 * c + 6] * inv, of[8 * c + 7] * inv);
-        dst[c] = w;
+        *reinterpret_cast<uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4)) = w;
+      }
+    }
+    __syncwarp();
+#pragma unroll 1
+    for (int q4 = 0; q4 < 8; ++q4) {
+      const int rr = 32 * warp + 4 * q4 + (lane >> 3), cc = lane & 7;
+      const int tk = q_begin + rr;
+      if (tk < q_end) {
+        const int ot = p.o_tok ? __ldg(p.o_tok + (size_t)b * p.n_patch + tk) : tk;
+        const uint4 w = *reinterpret_cast<const uint4*>(sQ + rr * 128 + ((cc ^ (rr & 7)) << 4));
+        *(reinterpret_cast<uint4*>(p.o + b * p.o_sb + (int64_t)(G + ot) * p.o_st + (int64_t)h * p.o_sh) + cc) = w;
       }
     }
   }
@@ -769,8 +794,10 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
     configured = true;
   }
   const int n_tok = plan->n_global + plan->n_patch;
-  CUtensorMap tq, tk, tv;
+  CUtensorMap tq, tk, tv, tkg, tvg;
   int32_t st;
+  if ((st = make_qkv_map(ctx, &tkg, io->k, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, plan->n_global)) != SPV_OK) return st;
+  if ((st = make_qkv_map(ctx, &tvg, io->v, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, plan->n_global)) != SPV_OK) return st;
   if ((st = make_qkv_map(ctx, &tq, io->q, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TQ)) != SPV_OK) return st;
   if ((st = make_qkv_map(ctx, &tk, io->k, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TK)) != SPV_OK) return st;
   if ((st = make_qkv_map(ctx, &tv, io->v, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TK)) != SPV_OK) return st;
@@ -785,7 +812,7 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   pp.status = ctx->d_status;
   const dim3 grid(plan->tiles_per_image, io->heads, plan->batch);
   SpvProfScope prof(ctx, SPV_K_ATTN_PATCH, stream);
-  attn_patch_kernel<<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, pp);
+  attn_patch_kernel<<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, tkg, tvg, pp);
   return spv_launch_ok(ctx);
 }
 
