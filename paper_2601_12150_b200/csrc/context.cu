@@ -132,8 +132,8 @@ extern "C" uint32_t spv_last_wait_site(const spv_ctx* ctx) { return ctx ? ctx->l
 
 extern "C" int64_t spv_launch_count(const spv_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
-int32_t spv_make_tmap_bf16(spv_ctx* ctx, CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
-                           const uint64_t* strides_bytes, const uint32_t* box) {
+static int32_t make_tmap(spv_ctx* ctx, CUtensorMap* map, CUtensorMapDataType dtype, const void* base, int rank,
+                         const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box) {
   if (((uintptr_t)base & 15u) != 0) return SPV_ERR_ALIGNMENT;
   cuuint64_t gdim[5];
   cuuint64_t gstr[4];
@@ -147,8 +147,18 @@ int32_t spv_make_tmap_bf16(spv_ctx* ctx, CUtensorMap* map, const void* base, int
       gstr[i - 1] = strides_bytes[i - 1];
     }
   }
-  CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, (void*)base, gdim, gstr,
-                                 bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+  CUresult r = ctx->encode_tiled(map, dtype, (cuuint32_t)rank, (void*)base, gdim, gstr, bx, es,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? SPV_OK : SPV_ERR_CUDA;
+}
+
+int32_t spv_make_tmap_bf16(spv_ctx* ctx, CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                           const uint64_t* strides_bytes, const uint32_t* box) {
+  return make_tmap(ctx, map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, base, rank, dims, strides_bytes, box);
+}
+
+int32_t spv_make_tmap_f32(spv_ctx* ctx, CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                          const uint64_t* strides_bytes, const uint32_t* box) {
+  return make_tmap(ctx, map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, base, rank, dims, strides_bytes, box);
 }

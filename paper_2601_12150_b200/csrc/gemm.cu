@@ -16,7 +16,8 @@ using namespace spv;
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
 constexpr int GEMM_THREADS = 192;
-constexpr int GEMM_SMEM = STAGES * (A_BYTES + B_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int EPI_BYTES = 128 * 128;    // one staging buffer: 128 rows x 128 bytes (32 fp32 or 64 bf16 columns)
+constexpr int GEMM_SMEM = STAGES * (A_BYTES + B_BYTES) + 2 * EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 
 struct EpiParams {
   void* out;
@@ -33,82 +34,62 @@ struct EpiParams {
 __device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
 __device__ __forceinline__ float silu(float x) { return x / (1.0f + __expf(-x)); }
 
+__host__ __device__ constexpr bool epi_is_f32(int epi) { return epi == SPV_EPI_BIAS_SCALE_RESID || epi == SPV_EPI_BIAS_ADDROW; }
+
+// Eight consecutive outputs of row m, columns n .. n+7 (accumulators in acc), with the epilogue
+// arithmetic applied; the result stays fp32.
 template <int EPI>
-__device__ __forceinline__ void epilogue_store(const EpiParams& p, int m, int n0, int n_total, const uint32_t* acc) {
-  // acc: 32 fp32 accumulators of row m, columns n0 .. n0+31
+__device__ __forceinline__ void epilogue_math(const EpiParams& p, int m, int n, const uint32_t* acc, float* v) {
 #pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    const int n = n0 + 8 * g;
-    if (n >= n_total) break;
-    float v[8];
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(acc[i]);
+  if (p.bias) {
+    const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + n));
+    const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + n + 4));
+    v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+    v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+  }
+  if constexpr (EPI == SPV_EPI_BIAS_GELU) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(acc[8 * g + i]);
-    if (p.bias) {
-      const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + n));
-      const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + n + 4));
-      v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
-      v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+    for (int i = 0; i < 8; ++i) v[i] = gelu_erf(v[i]);
+  } else if constexpr (EPI == SPV_EPI_BIAS_SILU) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = silu(v[i]);
+  } else if constexpr (EPI == SPV_EPI_BIAS_MUL) {
+    const uint4 a = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.aux) +
+                                                    (int64_t)m * p.ldaux + n);
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&aw[i]);
+      v[2 * i] *= __low2float(h);
+      v[2 * i + 1] *= __high2float(h);
     }
-    if constexpr (EPI == SPV_EPI_BIAS_GELU) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = gelu_erf(v[i]);
-    } else if constexpr (EPI == SPV_EPI_BIAS_SILU) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = silu(v[i]);
-    } else if constexpr (EPI == SPV_EPI_BIAS_MUL) {
-      const uint4 a = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.aux) +
-                                                      (int64_t)m * p.ldaux + n);
-      const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&aw[i]);
-        v[2 * i] *= __low2float(h);
-        v[2 * i + 1] *= __high2float(h);
-      }
+  } else if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID) {
+    if (p.scale) {
+      const float4 s0 = __ldg(reinterpret_cast<const float4*>(p.scale + n));
+      const float4 s1 = __ldg(reinterpret_cast<const float4*>(p.scale + n + 4));
+      v[0] *= s0.x; v[1] *= s0.y; v[2] *= s0.z; v[3] *= s0.w;
+      v[4] *= s1.x; v[5] *= s1.y; v[6] *= s1.z; v[7] *= s1.w;
     }
-    if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID || EPI == SPV_EPI_BIAS_ADDROW) {
-      float* o = reinterpret_cast<float*>(p.out) + (int64_t)m * p.ldo + n;
-      float4 r0, r1;
-      if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID) {
-        r0 = *reinterpret_cast<const float4*>(o);
-        r1 = *reinterpret_cast<const float4*>(o + 4);
-        float s[8] = {1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f};
-        if (p.scale) {
-          const float4 s0 = __ldg(reinterpret_cast<const float4*>(p.scale + n));
-          const float4 s1 = __ldg(reinterpret_cast<const float4*>(p.scale + n + 4));
-          s[0] = s0.x; s[1] = s0.y; s[2] = s0.z; s[3] = s0.w; s[4] = s1.x; s[5] = s1.y; s[6] = s1.z; s[7] = s1.w;
-        }
-        r0.x += s[0] * v[0]; r0.y += s[1] * v[1]; r0.z += s[2] * v[2]; r0.w += s[3] * v[3];
-        r1.x += s[4] * v[4]; r1.y += s[5] * v[5]; r1.z += s[6] * v[6]; r1.w += s[7] * v[7];
-      } else {
-        const float* ar = p.addrow + (int64_t)(m % p.rows_per_image) * p.ldadd + n;
-        const float4 a0 = __ldg(reinterpret_cast<const float4*>(ar));
-        const float4 a1 = __ldg(reinterpret_cast<const float4*>(ar + 4));
-        r0 = make_float4(v[0] + a0.x, v[1] + a0.y, v[2] + a0.z, v[3] + a0.w);
-        r1 = make_float4(v[4] + a1.x, v[5] + a1.y, v[6] + a1.z, v[7] + a1.w);
-      }
-      *reinterpret_cast<float4*>(o) = r0;
-      *reinterpret_cast<float4*>(o + 4) = r1;
-    } else {
-      uint4 w;
-      w.x = pack_bf16(v[0], v[1]);
-      w.y = pack_bf16(v[2], v[3]);
-      w.z = pack_bf16(v[4], v[5]);
-      w.w = pack_bf16(v[6], v[7]);
-      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)m * p.ldo + n) = w;
-    }
+  } else if constexpr (EPI == SPV_EPI_BIAS_ADDROW) {
+    const float* ar = p.addrow + (int64_t)(m % p.rows_per_image) * p.ldadd + n;
+    const float4 a0 = __ldg(reinterpret_cast<const float4*>(ar));
+    const float4 a1 = __ldg(reinterpret_cast<const float4*>(ar + 4));
+    v[0] += a0.x; v[1] += a0.y; v[2] += a0.z; v[3] += a0.w;
+    v[4] += a1.x; v[5] += a1.y; v[6] += a1.z; v[7] += a1.w;
   }
 }
 
 template <int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, int M, int N,
-                 int K, EpiParams ep, uint32_t* status) {
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+                 const __grid_constant__ CUtensorMap tm_out, int M, int N, int K, EpiParams ep, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
   uint8_t* sB = smem + STAGES * A_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_BYTES + B_BYTES));
+  uint8_t* sE = smem + STAGES * (A_BYTES + B_BYTES);     // [2] epilogue staging, 128-byte swizzle
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sE + 2 * EPI_BYTES);
   uint64_t* full = bars;                 // [STAGES]  TMA -> MMA
   uint64_t* empty = bars + STAGES;       // [STAGES]  MMA -> TMA
   uint64_t* acc_full = bars + 2 * STAGES;       // [2] MMA -> epilogue
@@ -176,26 +157,65 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       }
     }
   } else {
-    const int q = warp & 3;   // TMEM lane quadrant this warp may read
-    uint32_t tcount = 0;
+    // Epilogue: thread = output row.  A chunk of columns (32 fp32 or 64 bf16 = 128 bytes per row)
+    // goes TMEM -> registers -> arithmetic -> swizzled staging buffer, and one thread hands the
+    // buffer to TMA: a plain tile store, or an fp32 add into the residual stream, so that the
+    // residual is never read here and every global access is a whole 128-byte row segment.
+    constexpr bool F32 = epi_is_f32(EPI);
+    constexpr int CW = F32 ? 32 : 64;            // columns per chunk
+    const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+    const int row = q * 32 + lane;
+    const bool issuer = threadIdx.x == 64;
+    uint32_t tcount = 0, ec = 0;
     for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
       const int a = tcount & 1;
-      const int m = (tile % m_tiles) * BM + q * 32 + lane;
-      const int n_base = (tile / m_tiles) * BN;
+      const int m_base = (tile % m_tiles) * BM, n_base = (tile / m_tiles) * BN;
+      const int m = m_base + row;
       mbar_wait(&acc_full[a], (tcount >> 1) & 1, abort_flag, status, 0x400 + a);
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        if (n_base + c * 32 >= N) break;
-        uint32_t acc[32];
-        tmem_ld32(taddr + c * 32, acc);
+      for (int c = 0; c < BN / CW; ++c, ++ec) {
+        const int n0 = n_base + c * CW;
+        if (n0 >= N) break;
+        uint8_t* buf = sE + (ec & 1) * EPI_BYTES;
+        if (issuer) bulk_wait_read<1>();         // the store that last used this buffer has read it
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        uint32_t acc[CW];
+        tmem_ld32(taddr + c * CW, acc);
+        if constexpr (!F32) tmem_ld32(taddr + c * CW + 32, acc + 32);
         tc_wait_ld();
-        if (m < M) epilogue_store<EPI>(ep, m, n_base + c * 32, N, acc);
+#pragma unroll
+        for (int g = 0; g < CW / 8; ++g) {
+          float v[8];
+          if (m < M && n0 + 8 * g < N) {
+            epilogue_math<EPI>(ep, m, n0 + 8 * g, acc + 8 * g, v);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = 0.f;
+          }
+          if constexpr (F32) {
+            *reinterpret_cast<float4*>(buf + row * 128 + (((2 * g) ^ (row & 7)) << 4)) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4*>(buf + row * 128 + (((2 * g + 1) ^ (row & 7)) << 4)) = make_float4(v[4], v[5], v[6], v[7]);
+          } else {
+            uint4 w;
+            w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
+            w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
+            *reinterpret_cast<uint4*>(buf + row * 128 + ((g ^ (row & 7)) << 4)) = w;
+          }
+        }
+        fence_async_smem();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (issuer) {
+          if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID) tma_reduce_add_2d(&tm_out, buf, n0, m_base);
+          else tma_store_2d(&tm_out, buf, n0, m_base);
+          bulk_commit();
+        }
       }
       tc_fence_before();
       mbar_arrive(&acc_empty[a]);
     }
+    if (issuer) bulk_wait<0>();
   }
   tc_fence_before();
   __syncthreads();
@@ -206,6 +226,21 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 template <int EPI>
 int32_t launch(spv_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tw, const spv_gemm_desc* d, const EpiParams& ep,
                cudaStream_t stream) {
+  CUtensorMap tout;
+  {
+    const uint64_t dims[2] = {(uint64_t)d->n, (uint64_t)d->m};
+    int32_t st;
+    if (epi_is_f32(EPI)) {
+      const uint64_t str[1] = {(uint64_t)d->ldo * 4};
+      const uint32_t box[2] = {32, BM};
+      st = spv_make_tmap_f32(ctx, &tout, ep.out, 2, dims, str, box);
+    } else {
+      const uint64_t str[1] = {(uint64_t)d->ldo * 2};
+      const uint32_t box[2] = {64, BM};
+      st = spv_make_tmap_bf16(ctx, &tout, ep.out, 2, dims, str, box);
+    }
+    if (st != SPV_OK) return st;
+  }
   static bool configured = false;
   if (!configured) {
     SPV_CUDA_OK(cudaFuncSetAttribute(gemm_bf16_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
@@ -214,7 +249,7 @@ int32_t launch(spv_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tw, const
   const int tiles = ((d->m + BM - 1) / BM) * ((d->n + BN - 1) / BN);
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
   SpvProfScope prof(ctx, SPV_K_GEMM, stream, 2.0 * (double)d->m * (double)d->n * (double)d->k);
-  gemm_bf16_kernel<EPI><<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tw, d->m, d->n, d->k, ep, ctx->d_status);
+  gemm_bf16_kernel<EPI><<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tw, tout, d->m, d->n, d->k, ep, ctx->d_status);
   return spv_launch_ok(ctx);
 }
 
