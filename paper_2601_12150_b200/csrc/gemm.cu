@@ -5,8 +5,10 @@
 //   warp 0      TMA producer (A and W slices, 128-byte swizzle, 4-stage ring)
 //   warp 1      tcgen05.mma issuer (one thread), owns the TMEM allocation (2 x 256 columns, so
 //               the epilogue of tile i overlaps the main loop of tile i+1)
-//   warps 2..5  epilogue: TMEM -> registers -> bias / activation / residual -> global
-// Rows beyond M and columns beyond N are zero-filled by TMA on load and predicated on store.
+//   warps 2..9  epilogue, two threads per output row: TMEM -> registers -> bias / activation /
+//               scale -> swizzled staging buffer -> TMA tile store (bf16 outputs, fp32 rows) or
+//               fp32 TMA add-reduce into the residual stream
+// Rows beyond M and columns beyond N are zero-filled by TMA on load and clipped by TMA on store.
 #include "common.cuh"
 
 namespace {
@@ -15,7 +17,8 @@ using namespace spv;
 
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 320;      // warp 0 TMA, warp 1 MMA, warps 2-9 epilogue (two per TMEM lane quadrant)
+constexpr int EPI_THREADS = 256;
 constexpr int EPI_BYTES = 128 * 128;    // one staging buffer: 128 rows x 128 bytes (32 fp32 or 64 bf16 columns)
 constexpr int GEMM_SMEM = STAGES * (A_BYTES + B_BYTES) + 2 * EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 
@@ -104,7 +107,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 128); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], EPI_THREADS); }
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -163,7 +166,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     // residual is never read here and every global access is a whole 128-byte row segment.
     constexpr bool F32 = epi_is_f32(EPI);
     constexpr int CW = F32 ? 32 : 64;            // columns per chunk
+    constexpr int TW = CW / 2;                   // columns per thread: two threads share a row
     const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+    const int half = (warp - 2) >> 2;            // which half of the chunk's columns
     const int row = q * 32 + lane;
     const bool issuer = threadIdx.x == 64;
     uint32_t tcount = 0, ec = 0;
@@ -180,32 +185,34 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         if (n0 >= N) break;
         uint8_t* buf = sE + (ec & 1) * EPI_BYTES;
         if (issuer) bulk_wait_read<1>();         // the store that last used this buffer has read it
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        uint32_t acc[CW];
-        tmem_ld32(taddr + c * CW, acc);
-        if constexpr (!F32) tmem_ld32(taddr + c * CW + 32, acc + 32);
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        uint32_t acc[TW];
+        if constexpr (F32) tmem_ld16(taddr + c * CW + half * TW, acc);
+        else tmem_ld32(taddr + c * CW + half * TW, acc);
         tc_wait_ld();
 #pragma unroll
-        for (int g = 0; g < CW / 8; ++g) {
+        for (int g = 0; g < TW / 8; ++g) {
           float v[8];
-          if (m < M && n0 + 8 * g < N) {
-            epilogue_math<EPI>(ep, m, n0 + 8 * g, acc + 8 * g, v);
+          const int n = n0 + half * TW + 8 * g;
+          if (m < M && n < N) {
+            epilogue_math<EPI>(ep, m, n, acc + 8 * g, v);
           } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = 0.f;
           }
           if constexpr (F32) {
-            *reinterpret_cast<float4*>(buf + row * 128 + (((2 * g) ^ (row & 7)) << 4)) = make_float4(v[0], v[1], v[2], v[3]);
-            *reinterpret_cast<float4*>(buf + row * 128 + (((2 * g + 1) ^ (row & 7)) << 4)) = make_float4(v[4], v[5], v[6], v[7]);
+            const int c16 = 4 * half + 2 * g;
+            *reinterpret_cast<float4*>(buf + row * 128 + ((c16 ^ (row & 7)) << 4)) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4*>(buf + row * 128 + (((c16 + 1) ^ (row & 7)) << 4)) = make_float4(v[4], v[5], v[6], v[7]);
           } else {
             uint4 w;
             w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
             w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
-            *reinterpret_cast<uint4*>(buf + row * 128 + ((g ^ (row & 7)) << 4)) = w;
+            *reinterpret_cast<uint4*>(buf + row * 128 + (((4 * half + g) ^ (row & 7)) << 4)) = w;
           }
         }
         fence_async_smem();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (issuer) {
           if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID) tma_reduce_add_2d(&tm_out, buf, n0, m_base);
           else tma_store_2d(&tm_out, buf, n0, m_base);
