@@ -214,6 +214,12 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 __device__ __forceinline__ void unpack8(const uint4& u, float* f) {
   const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
@@ -446,13 +452,13 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if (32 * c < u_hi && 32 * c + 32 > u_lo) {
             float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              m0 = fmaxf(m0, __uint_as_float(sr[32 * c + i]));
-              m1 = fmaxf(m1, __uint_as_float(sr[32 * c + i + 1]));
-              m2 = fmaxf(m2, __uint_as_float(sr[32 * c + i + 2]));
-              m3 = fmaxf(m3, __uint_as_float(sr[32 * c + i + 3]));
+            for (int i = 0; i < 32; i += 8) {
+              m0 = fmax3(m0, __uint_as_float(sr[32 * c + i]), __uint_as_float(sr[32 * c + i + 1]));
+              m1 = fmax3(m1, __uint_as_float(sr[32 * c + i + 2]), __uint_as_float(sr[32 * c + i + 3]));
+              m2 = fmax3(m2, __uint_as_float(sr[32 * c + i + 4]), __uint_as_float(sr[32 * c + i + 5]));
+              m3 = fmax3(m3, __uint_as_float(sr[32 * c + i + 6]), __uint_as_float(sr[32 * c + i + 7]));
             }
-            mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
+            mx = fmax3(mx, fmaxf(m0, m1), fmaxf(m2, m3));
           }
         }
         // lazy rescale: the running maximum only moves when it would grow by more than 2^8
@@ -478,18 +484,25 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
         // p = 2^(s*scale - m) chunk by chunk, packed to bf16 pairs and written to TMEM at once
         // (masked scores are -inf, so p = 0)
-        float rs0 = 0.f, rs1 = 0.f;
+        // (two scores per packed fp32x2 multiply-add and per packed add)
+        float2 rs_a = make_float2(0.f, 0.f), rs_b = make_float2(0.f, 0.f);
+        const float2 sl2_2 = make_float2(sl2, sl2), nm_2 = make_float2(-m_new, -m_new);
 #pragma unroll
         for (int c = 0; c < TK / 32; ++c) {
           uint32_t pk[16];
           if (32 * c < u_hi && 32 * c + 32 > u_lo) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const float p0 = fast_exp2(fmaf(__uint_as_float(sr[32 * c + i]), sl2, -m_new));
-              const float p1 = fast_exp2(fmaf(__uint_as_float(sr[32 * c + i + 1]), sl2, -m_new));
-              rs0 += p0;
-              rs1 += p1;
-              pk[i / 2] = pack_bf16(p0, p1);
+            for (int i = 0; i < 32; i += 4) {
+              const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(sr[32 * c + i]), __uint_as_float(sr[32 * c + i + 1])),
+                                           sl2_2, nm_2);
+              const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(sr[32 * c + i + 2]), __uint_as_float(sr[32 * c + i + 3])),
+                                           sl2_2, nm_2);
+              const float2 p0 = make_float2(fast_exp2(x0.x), fast_exp2(x0.y));
+              const float2 p1 = make_float2(fast_exp2(x1.x), fast_exp2(x1.y));
+              rs_a = __fadd2_rn(rs_a, p0);
+              rs_b = __fadd2_rn(rs_b, p1);
+              pk[i / 2] = pack_bf16(p0.x, p0.y);
+              pk[i / 2 + 1] = pack_bf16(p1.x, p1.y);
             }
           } else {
 #pragma unroll
@@ -497,7 +510,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           }
           tmem_st16(lane_addr + P_COL + 16 * c, pk);
         }
-        l = l * alpha + (rs0 + rs1);
+        l = l * alpha + ((rs_a.x + rs_a.y) + (rs_b.x + rs_b.y));
         m = m_new;
         tc_wait_st();
         tc_fence_before();
