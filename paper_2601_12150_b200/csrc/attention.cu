@@ -380,18 +380,15 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       }
 #pragma unroll 1
       for (int g = 0; g < G; ++g) {
-        float d0 = 0.f, d1 = 0.f;
+        float d[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};     // eight independent chains
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           float kf[8];
           unpack8(*reinterpret_cast<const uint4*>(sKg + g * 128 + ((c ^ (g & 7)) << 4)), kf);
 #pragma unroll
-          for (int i = 0; i < 8; i += 2) {
-            d0 = fmaf(qf[8 * c + i], kf[i], d0);
-            d1 = fmaf(qf[8 * c + i + 1], kf[i + 1], d1);
-          }
+          for (int i = 0; i < 8; ++i) d[i] = fmaf(qf[8 * c + i], kf[i], d[i]);
         }
-        const float sc = (d0 + d1) * sl2;
+        const float sc = (((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]))) * sl2;
         s_sg[g * 128 + row] = sc;
         m = fmaxf(m, sc);
       }
@@ -425,6 +422,8 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tc_fence_after();
         // boundary chunks (some of the warp's rows see only part of them) are masked in place
         // first, by a small loop, so that the unrolled main pass below carries no mask code
+        // (none exist when every live chunk lies inside the intersection)
+        if (((u_lo & ~31) < i_lo) || (((u_hi + 31) & ~31) > i_hi)) {
 #pragma unroll 1
         for (int cb = 0; cb < TK; cb += 32) {
           if (cb < u_hi && cb + 32 > u_lo && !(cb >= i_lo && cb + 32 <= i_hi)) {
@@ -438,6 +437,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           }
         }
         tc_wait_st();
+        }
         // one pass: the live 32-column chunks of S go to registers, then S is released
         uint32_t sr[TK];
 #pragma unroll
@@ -562,15 +562,20 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       }
     }
     __syncwarp();
-#pragma unroll 1
-    for (int q4 = 0; q4 < 8; ++q4) {
-      const int rr = 32 * warp + 4 * q4 + (lane >> 3), cc = lane & 7;
-      const int tk = q_begin + rr;
-      if (tk < q_end) {
-        const int ot = p.o_tok ? __ldg(p.o_tok + (size_t)b * p.n_patch + tk) : tk;
-        const uint4 w = *reinterpret_cast<const uint4*>(sQ + rr * 128 + ((cc ^ (rr & 7)) << 4));
-        *(reinterpret_cast<uint4*>(p.o + b * p.o_sb + (int64_t)(G + ot) * p.o_st + (int64_t)h * p.o_sh) + cc) = w;
+    {
+      const int r0 = 32 * warp + (lane >> 3), cc = lane & 7;
+      __nv_bfloat16* obase = p.o + b * p.o_sb + (int64_t)G * p.o_st + (int64_t)h * p.o_sh + cc * 8;
+      uint4 w[8];
+      int ot[8];
+#pragma unroll
+      for (int q4 = 0; q4 < 8; ++q4) {
+        const int rr = r0 + 4 * q4, tk = q_begin + rr;
+        w[q4] = *reinterpret_cast<const uint4*>(sQ + rr * 128 + ((cc ^ (rr & 7)) << 4));
+        ot[q4] = (p.o_tok && tk < q_end) ? __ldg(p.o_tok + (size_t)b * p.n_patch + tk) : tk;
       }
+#pragma unroll
+      for (int q4 = 0; q4 < 8; ++q4)
+        if (q_begin + r0 + 4 * q4 < q_end) *reinterpret_cast<uint4*>(obase + (int64_t)ot[q4] * p.o_st) = w[q4];
     }
   }
   tc_fence_before();
