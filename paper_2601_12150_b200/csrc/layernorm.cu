@@ -5,9 +5,10 @@
 
 namespace {
 
-constexpr int kMaxVec = 16;   // float4 per lane held in registers: dim <= 2048
-
-__global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict__ x, int64_t rows, int dim,
+// kMaxVec float4 per lane are held in registers (dim <= 128 * kMaxVec); the instantiation that just
+// covers the row keeps the register count low, so that more warps (more loads in flight) fit an SM.
+template <int kMaxVec>
+__global__ void __launch_bounds__(256, (kMaxVec <= 8 ? 3 : 2)) layernorm_kernel(const float* __restrict__ x, int64_t rows, int dim,
                                                         const float* __restrict__ gamma,
                                                         const float* __restrict__ beta, float eps,
                                                         __nv_bfloat16* __restrict__ y,
@@ -88,10 +89,15 @@ extern "C" int32_t spv_layernorm(spv_ctx* ctx, const float* x, int64_t rows, int
   if (((uintptr_t)x & 15u) || ((uintptr_t)y & 15u) || ((uintptr_t)gamma & 15u) || ((uintptr_t)beta & 15u))
     return SPV_ERR_ALIGNMENT;
   int64_t blocks = (rows + 7) / 8;
-  const int64_t cap = (int64_t)ctx->sm_count * 8;
+  const int64_t cap = (int64_t)ctx->sm_count * 64;
   if (blocks > cap) blocks = cap;
   SpvProfScope prof(ctx, SPV_K_LAYERNORM, (cudaStream_t)stream, (double)rows * dim * 6.0);
-  layernorm_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(x, rows, dim, gamma, beta, eps,
-                                                                      (__nv_bfloat16*)y, out_row);
+  const unsigned g = (unsigned)blocks;
+  cudaStream_t st = (cudaStream_t)stream;
+  __nv_bfloat16* yo = (__nv_bfloat16*)y;
+  if (dim <= 512) layernorm_kernel<4><<<g, 256, 0, st>>>(x, rows, dim, gamma, beta, eps, yo, out_row);
+  else if (dim <= 1024) layernorm_kernel<8><<<g, 256, 0, st>>>(x, rows, dim, gamma, beta, eps, yo, out_row);
+  else if (dim <= 1536) layernorm_kernel<12><<<g, 256, 0, st>>>(x, rows, dim, gamma, beta, eps, yo, out_row);
+  else layernorm_kernel<16><<<g, 256, 0, st>>>(x, rows, dim, gamma, beta, eps, yo, out_row);
   return spv_launch_ok(ctx);
 }
