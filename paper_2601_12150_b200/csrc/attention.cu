@@ -611,6 +611,7 @@ __global__ void __launch_bounds__(256) attn_global_partial(const __nv_bfloat16* 
   float lmax = -INFINITY;
   // the trip count is the same for every lane (the shuffles name the whole warp); keys past the
   // end of the chunk are predicated off
+#pragma unroll 4
   for (int kk0 = k0; kk0 < k1; kk0 += 32) {
     const int kk = kk0 + grp;
     const bool live = kk < k1;
@@ -649,6 +650,7 @@ __global__ void __launch_bounds__(256) attn_global_partial(const __nv_bfloat16* 
   __syncthreads();
   if ((threadIdx.x & 31) == 0) s_red[8 + (threadIdx.x >> 5)] = lsum;
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
   for (int kk = k0 + grp; kk < k1; kk += 32) {
     const float pw = __expf(s_s[kk - k0] - cmax);
     float vf[8];
