@@ -10,7 +10,7 @@
 //
 // Kernels
 //   attn_plan_*        per-block token counts (binary search in the sorted positions), scan,
-//                      greedy packing of consecutive blocks into <=128-row query tiles
+//                      each block row cut into 128-row query tiles
 //   attn_regroup       row-major -> block-major copy of Q, K, V (only for row-major callers)
 //   attn_patch_kernel  flash-style tcgen05 kernel: S = Q K^T into TMEM, online softmax by 128
 //                      row-owning threads, P written back to TMEM as bf16, O += P V with V as an
@@ -95,9 +95,7 @@ __global__ void attn_plan_segments(SpvAttnPlan p, const int32_t* __restrict__ pa
   p.seg_cnt[(size_t)b * p.nseg + seg] = cnt;
 }
 
-// One CTA per image: exclusive scan of the segment counts, block offsets, then the query tiles:
-// per block row, consecutive blocks are packed greedily into tiles of at most TQ tokens; a block
-// larger than TQ is cut into TQ-row pieces.
+// One CTA per image: exclusive scan of the segment counts, block offsets, then the query tiles.
 __global__ void __launch_bounds__(1024) attn_plan_scan(SpvAttnPlan p) {
   __shared__ int warp_sums[32];
   __shared__ int carry;
@@ -133,21 +131,22 @@ __global__ void __launch_bounds__(1024) attn_plan_scan(SpvAttnPlan p) {
   int32_t* boff = p.block_off + (size_t)b * (p.nb + 1);
   for (int blk = threadIdx.x; blk <= p.nb; blk += 1024) boff[blk] = off[min(blk * p.segs_per_block, p.nseg)];
   __syncthreads();
+  // query tiles: the tokens of one block row cut into runs of TQ (a block may straddle two tiles;
+  // every row looks up its own block), each with the first and last block it touches
   int4* tiles = p.tiles + (size_t)b * p.tiles_per_image;
   for (int by = threadIdx.x; by < p.nby; by += 1024) {
     int4* t = tiles + (size_t)by * p.tiles_per_row;
     int nt = 0;
-    int cur_begin = -1, cur_end = 0, cur_first = 0, cur_last = 0;
-    for (int bx = 0; bx < p.nbx; ++bx) {
-      int s = boff[by * p.nbx + bx];
-      const int e = boff[by * p.nbx + bx + 1];
-      if (e == s) continue;
-      if (cur_begin >= 0 && (e - cur_begin) <= TQ) { cur_end = e; cur_last = bx; continue; }
-      if (cur_begin >= 0) { t[nt++] = make_int4(cur_begin, cur_end, by, cur_first | (cur_last << 16)); cur_begin = -1; }
-      while (e - s > TQ) { t[nt++] = make_int4(s, s + TQ, by, bx | (bx << 16)); s += TQ; }
-      cur_begin = s; cur_end = e; cur_first = bx; cur_last = bx;
+    const int row_end = boff[(by + 1) * p.nbx];
+    int bx = 0;
+    for (int s = boff[by * p.nbx]; s < row_end; s += TQ) {
+      const int e = min(s + TQ, row_end);
+      while (boff[by * p.nbx + bx + 1] <= s) ++bx;
+      const int first = bx;
+      int last = bx;
+      while (boff[by * p.nbx + last + 1] < e) ++last;
+      t[nt++] = make_int4(s, e, by, first | (last << 16));
     }
-    if (cur_begin >= 0) t[nt++] = make_int4(cur_begin, cur_end, by, cur_first | (cur_last << 16));
     for (; nt < p.tiles_per_row; ++nt) t[nt] = make_int4(0, 0, 0, 0);
   }
 }
@@ -755,10 +754,7 @@ static void plan_geometry(SpvAttnPlan* p, int token_order) {
   p->segs_per_block = token_order == SPV_TOKENS_ROW_MAJOR ? p->block : 1;
   p->nseg = p->nb * p->segs_per_block;
   const int64_t rowcap = (int64_t)(p->block < p->grid_h ? p->block : p->grid_h) * p->grid_w;
-  const int64_t full = (rowcap + TQ - 1) / TQ;
-  int64_t t = 2 * full + 1;
-  if (p->nbx + full < t) t = p->nbx + full;
-  p->tiles_per_row = (int32_t)t;
+  p->tiles_per_row = (int32_t)((rowcap + TQ - 1) / TQ);
   p->tiles_per_image = p->tiles_per_row * p->nby;
   p->identity = token_order == SPV_TOKENS_BLOCK_MAJOR;
 }
