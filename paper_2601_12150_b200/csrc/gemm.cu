@@ -126,7 +126,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       tma_prefetch_desc(&tm_w);
       uint32_t it = 0;
       for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-        const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+        // column tile fastest: the CTAs running together share a few row tiles of A and all of W in L2,
+        // so A crosses HBM once instead of once per column tile
+        const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % STAGES;
           mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, status, 0x100 + s);
@@ -174,7 +176,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     uint32_t tcount = 0, ec = 0;
     for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
       const int a = tcount & 1;
-      const int m_base = (tile % m_tiles) * BM, n_base = (tile / m_tiles) * BN;
+      const int m_base = (tile / n_tiles) * BM, n_base = (tile % n_tiles) * BN;
       const int m = m_base + row;
       mbar_wait(&acc_full[a], (tcount >> 1) & 1, abort_flag, status, 0x400 + a);
       tc_fence_after();
