@@ -34,7 +34,25 @@ struct EpiParams {
   int32_t rows_per_image;
 };
 
-__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+// Exact (erf) GELU.  erf by the rational/exponential form of Abramowitz & Stegun 7.1.26
+// (|error| <= 1.5e-7, branch-free: one reciprocal, one exponential, five multiply-adds), which keeps
+// the epilogue of the MLP GEMM shorter than its main loop; the absolute error of the GELU value is
+// below |x| * 1e-7, far inside the bf16 rounding of the stored activation.
+__device__ __forceinline__ float gelu_erf(float x) {
+  const float z = fabsf(x) * 0.70710678118654752f;
+  float t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, z, 1.0f)));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  poly *= t;
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(z * z * -1.4426950408889634f));
+  const float erf_abs = fmaf(-poly, e, 1.0f);           // erf(|x| / sqrt 2)
+  const float half_x = 0.5f * x;
+  return fmaf(fabsf(half_x), erf_abs, half_x);          // 0.5 x (1 + sign(x) erf(|x|/sqrt 2))
+}
 __device__ __forceinline__ float silu(float x) { return x / (1.0f + __expf(-x)); }
 
 __host__ __device__ constexpr bool epi_is_f32(int epi) { return epi == SPV_EPI_BIAS_SCALE_RESID || epi == SPV_EPI_BIAS_ADDROW; }
