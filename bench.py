@@ -289,12 +289,13 @@ def run_gpu(args, wl, rank, world):
     ctx.check()
     kept_host = kept.cpu().numpy() if kept is not None else None
 
-    # ---- timed region: device-resident inputs, per-class event timing on
+    # ---- timed region: device-resident inputs.  K steps timed as a whole give `value`; the same K
+    # steps are then repeated with the library's per-launch CUDA events switched on, which gives the
+    # per-class times of the roofline figures (the events cost a little, so they stay out of `value`).
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
     barrier()
     sampler.start()
     launches0 = ctx.launch_count()
-    ctx.profile(True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record(stream)
@@ -304,27 +305,54 @@ def run_gpu(args, wl, rank, world):
     barrier()
     ms = e0.elapsed_time(e1)
     launches = ctx.launch_count() - launches0
+    ctx.profile(True)
+    for _ in range(args.steps):
+        step()
     prof = ctx.profile_read()
     ctx.profile(False)
     ctx.check()
     clocks = sampler.stop()
     peak_bytes = torch.cuda.max_memory_allocated()
 
-    # ---- end to end: pinned host images in, output tokens back to the host, every step
-    def e2e_step():
-        img.copy_(img_host, non_blocking=True)
-        step()
-        out_host.copy_(out, non_blocking=True)
-
+    # ---- end to end: pinned host images in, output tokens back to the host, every step.  The way a
+    # user of the library would run a stream of batches: copies on their own streams, double-buffered,
+    # so that the copy of batch i+1 and the read-back of batch i-1 overlap the forward of batch i.
+    # Every byte of every step is copied inside the timed region.
     ms_e2e = float("nan")
     if not args.quick:
-        for _ in range(2):
-            e2e_step()
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        imgs = [img, torch.empty_like(img)]
+        outs = [out, torch.empty_like(out)]
+        outs_host = [out_host, torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()]
+        in_ready = [torch.cuda.Event() for _ in range(2)]
+        comp_done = [torch.cuda.Event() for _ in range(2)]
+        out_done = [torch.cuda.Event() for _ in range(2)]
+
+        def e2e_run(n):
+            for i in range(n):
+                bsel = i & 1
+                with torch.cuda.stream(s_in):
+                    if i >= 2:
+                        s_in.wait_event(comp_done[bsel])          # the forward that read this buffer is done
+                    imgs[bsel].copy_(img_host, non_blocking=True)
+                    in_ready[bsel].record(s_in)
+                stream.wait_event(in_ready[bsel])
+                if i >= 2:
+                    stream.wait_event(out_done[bsel])             # its previous result has been read back
+                ctx.vit_forward(c, dw, imgs[bsel], g, g, out=outs[bsel])
+                comp_done[bsel].record(stream)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(comp_done[bsel])
+                    outs_host[bsel].copy_(outs[bsel], non_blocking=True)
+                    out_done[bsel].record(s_out)
+            stream.wait_event(out_done[0])
+            stream.wait_event(out_done[1])
+
+        e2e_run(2)
         barrier()
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record(stream)
-        for _ in range(args.steps):
-            e2e_step()
+        e2e_run(args.steps)
         f1.record(stream)
         barrier()
         ms_e2e = f0.elapsed_time(f1)

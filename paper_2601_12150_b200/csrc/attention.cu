@@ -599,7 +599,8 @@ __global__ void __launch_bounds__(256) attn_global_partial(const __nv_bfloat16* 
   __shared__ float s_s[GCH];
   __shared__ float s_red[32];
   __shared__ float s_o[32][HD + 1];
-  const int chunk = blockIdx.x, h = blockIdx.y, bg = blockIdx.z;
+  // heads fastest: the CTAs running together read whole token rows (all heads) of one key chunk
+  const int h = blockIdx.x, chunk = blockIdx.y, bg = blockIdx.z;
   const int b = bg / n_global, g = bg % n_global;
   const int k0 = chunk * GCH, k1 = min(k0 + GCH, n_tok);
   const int sub = threadIdx.x & 7, grp = threadIdx.x >> 3;   // 8 lanes per key, 32 keys in flight
@@ -850,7 +851,7 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   float* part_ml = (float*)w; w += spv_align_up(rows * chunks * 2 * 4, 256);
   float* part_o = (float*)w;
   SpvProfScope prof(ctx, SPV_K_ATTN_GLOBAL, stream);
-  attn_global_partial<<<dim3(chunks, io->heads, B * G), 256, 0, stream>>>(
+  attn_global_partial<<<dim3(io->heads, chunks, B * G), 256, 0, stream>>>(
       (const __nv_bfloat16*)io->q, (const __nv_bfloat16*)io->k, (const __nv_bfloat16*)io->v, io->sb, io->st, io->sh,
       n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks);
   attn_global_combine<<<dim3(io->heads, B * G), 256, 0, stream>>>(logits, part_ml, part_o, chunks, n_tok, G,
