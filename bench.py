@@ -247,6 +247,26 @@ def run_reference(args, wl, rank):
 
 
 # --------------------------------------------------------------------------------------------
+# multi-rank bookkeeping (replicas only: the path has no exchange step, so the only collective is
+# this reduction of the timings)
+# --------------------------------------------------------------------------------------------
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of a list of floats over all ranks (identity when world == 1)."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    tt = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return tt.tolist()
+
+
+def whole_job_rate(units_per_rank, world, ms):
+    """Units per second of the whole job: every rank processed `units_per_rank` in `ms` (max over ranks)."""
+    return units_per_rank * world / (ms * 1e-3)
+
+
+# --------------------------------------------------------------------------------------------
 # GPU arm
 # --------------------------------------------------------------------------------------------
 def run_gpu(args, wl, rank, world):
@@ -358,10 +378,7 @@ def run_gpu(args, wl, rank, world):
         ms_e2e = f0.elapsed_time(f1)
         ctx.check()
 
-    if world > 1:
-        tt = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = tt.tolist()
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], world, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -369,7 +386,7 @@ def run_gpu(args, wl, rank, world):
 
     pk = peaks()
     images = B * args.steps * world
-    value = images / (ms * 1e-3)
+    value = whole_job_rate(B * args.steps, world, ms)
     fl = forward_flops(wl, kept_host)
     steps = args.steps
     tot_ms = sum(v["ms"] for v in prof.values()) or 1.0

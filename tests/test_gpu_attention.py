@@ -147,3 +147,32 @@ def test_sampled_rows_at_full_size(ctx):
     want, wsc = oracle.attention(q, k, v, gh, gw, 8, 1, rows=rows, want_scores=True)
     _check(got[:, rows], want[:, rows])
     assert np.abs(gsc - wsc).max() < 1e-3
+
+
+def test_sampled_rows_146_grid_radius_2(ctx):
+    """ViT-g/14-style geometry: 146x146 grid (19x19 blocks, the last row/column 2 patches wide), 5x5
+    neighbourhood, 21317 tokens; sampled query rows (first, last, edge blocks) against the oracle."""
+    gh = gw = 146
+    q, k, v = synth.attention_qkv(4, 1, 1 + gh * gw, 3, 64)
+    got, gsc = _run(ctx, q, k, v, gh, gw, 8, 2, packed=True)
+    rng = np.random.default_rng(1)
+    edge = [1 + y * gw + x for y in (0, 143, 144, 145) for x in (0, 7, 8, 143, 144, 145)]
+    rows = np.unique(np.concatenate([[0, 1, gh * gw], edge, rng.integers(1, 1 + gh * gw, size=200)])).astype(np.int32)
+    want, wsc = oracle.attention(q, k, v, gh, gw, 8, 2, rows=rows, want_scores=True)
+    _check(got[:, rows], want[:, rows])
+    assert np.abs(gsc - wsc).max() < 1e-3
+
+
+def test_sampled_rows_filtered_full_size(ctx):
+    """128x128 grid with half of the tokens kept at scattered positions (what the filter leaves
+    behind with random weights), block-major order as inside vit_forward; sampled rows."""
+    gh = gw = 128
+    rng = np.random.default_rng(2)
+    kept = np.sort(rng.choice(gh * gw, size=8192, replace=False))
+    order = np.lexsort((kept, (kept % gw) // 8, (kept // gw) // 8))
+    pos_bm = kept[order].astype(np.int32)[None]
+    q, k, v = synth.attention_qkv(5, 1, 1 + 8192, 2, 64)
+    got, _ = _run(ctx, q, k, v, gh, gw, 8, 1, patch_pos=pos_bm, order=1, scores=False)
+    rows = np.unique(np.concatenate([[0, 1, 8192], rng.integers(1, 8193, size=250)])).astype(np.int32)
+    want, _ = oracle.attention(q, k, v, gh, gw, 8, 1, patch_pos=pos_bm, rows=rows)
+    _check(got[:, rows], want[:, rows])
