@@ -125,6 +125,15 @@ def test_vit_forward_wide_model_layer_growth(ctx):
     _compare(ctx, arch, cfg, 16, 16, 1, seed=2)
 
 
+def test_vit_forward_g14_style_block_shapes(ctx):
+    """d = 1536, 24 heads, SwiGLU hidden 4096, patch 14 (im2col width 588, padded to 592), no
+    LayerScale: the ViT-g/14-style block shapes on a ragged 18x11 grid, 5x5 neighbourhood, 2 layers
+    with the filter after block 1."""
+    arch = dict(synth.vit_g14(), layers=2)
+    cfg = dict(attn_mode=synth.ATTN_SPARSE, block=8, radius=2, filter_layer=1, keep_ratio=0.5)
+    _compare(ctx, arch, cfg, 18, 11, 1, seed=4)
+
+
 def test_vit_forward_argument_errors(ctx):
     import paper_2601_12150_b200 as spv
     arch = synth.vit_tiny(layers=1, dim=128, heads=2, hidden=256, patch=4)
