@@ -115,7 +115,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // then runs to its normal end (its loops are bounded by tile counts), releases TMEM and exits;
 // the host reads the status through spv_check().
 #ifndef SPV_WAIT_LIMIT_NS
-#define SPV_WAIT_LIMIT_NS 1000000000ull
+#define SPV_WAIT_LIMIT_NS 1000000000u
 #endif
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
@@ -138,16 +138,22 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t par
 }
 static __device__ __forceinline__ void mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
                                                       uint32_t* status, uint32_t site) {
-  const uint64_t t0 = global_ns();
+  // kept short on purpose: this body is inlined at every wait of the big kernels, and their
+  // instruction footprint costs more than a few nanoseconds of timer precision (32-bit timer:
+  // limits below four seconds)
+  uint32_t t0;
+  asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t0));
   for (;;) {
     if (mbar_try_wait_parked(bar, parity, 20000u)) return;
-    if (*abort_flag) return;
-    // another CTA already gave up: do not wait out a second limit here
-    if (*reinterpret_cast<volatile uint32_t*>(status) != 0u) { *abort_flag = 1; return; }
-    if (global_ns() - t0 > SPV_WAIT_LIMIT_NS) break;
+    uint32_t t;
+    asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t));
+    // give up when this CTA or any other CTA of the grid already has, or when the limit is reached
+    if ((*abort_flag | *reinterpret_cast<volatile uint32_t*>(status)) != 0u || t - t0 > (uint32_t)SPV_WAIT_LIMIT_NS) break;
   }
-  *abort_flag = 1;
-  atomicCAS(status, 0u, site);
+  if (*abort_flag == 0u) {
+    *abort_flag = 1;
+    atomicCAS(status, 0u, site);
+  }
 }
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           uint32_t* status, uint32_t site) {
