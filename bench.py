@@ -91,6 +91,25 @@ def forward_flops(wl, kept_positions):
     return dict(gemm=gemm, attn_patch=attn_patch, attn_global=attn_glob)
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per GEMM launch, averaged over the 104
+# GEMM launches of one step, from one ncu capture (profiles/gemm_dram_vitl16_2048_b4.md).  Valid
+# only for the kernel source it was taken with: reported as null once gemm.cu has changed.
+GEMM_TRAFFIC = {"vitl16_2048_b4_sparse_filter": (384.3e6, "ee14d77817d5")}
+
+
+def gemm_traffic(workload):
+    import hashlib
+    ent = GEMM_TRAFFIC.get(workload)
+    if ent is None:
+        return None
+    src = os.path.join(ROOT, "paper_2601_12150_b200", "csrc", "gemm.cu")
+    try:
+        sha = hashlib.sha1(open(src, "rb").read()).hexdigest()[:12]
+    except OSError:
+        return None
+    return ent[0] if sha == ent[1] else None
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -409,7 +428,8 @@ def run_gpu(args, wl, rank, world):
     top = max(brk, key=lambda n: brk[n]["share"])
     roof = {"kernel": top, "bound": brk[top].get("bound"), "achieved": brk[top].get("achieved"),
             "peak": brk[top].get("peak"), "unit": "TFLOP/s" if brk[top].get("bound") == "tensor" else "GB/s",
-            "frac": brk[top].get("frac"), "traffic": None,
+            "frac": brk[top].get("frac"),
+            "traffic": gemm_traffic(wl["name"]) if top == "gemm" else None,
             "peak_source": f"of {pk['source']} (sustained bf16 figure: the kernel is timed inside a long step)"}
     total_flops = fl["gemm"] + fl["attn_patch"] + fl["attn_global"]
     line = {
