@@ -461,6 +461,60 @@ def run_gpu(args, wl, rank, world):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------------------------
+# resolution sweep (ViT-L/16, batch 4): dense attention, neighbour-block sparse, sparse + filter
+# --------------------------------------------------------------------------------------------
+def run_sweep(args):
+    """One JSON line per (image side, mode): images/s, peak HBM bytes, useful TFLOP/s and its fraction
+    of the measured bf16 peak.  Dense attention is the same kernel with a radius that covers the grid."""
+    import torch
+    import paper_2601_12150_b200 as spv
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = spv.Context(0)
+    pk = peaks()
+    arch = synth.vit_l16()
+    B = 4
+    sides = [int(x) for x in args.sweep_sides.split(",")]
+    for side in sides:
+        g = side // arch["patch"]
+        w = synth.vit_weights(2, arch, g, g)
+        dw = ctx.make_vit_weights(w)
+        del w
+        img = torch.from_numpy(synth.tissue_batch(6, B, side, side, background_range=(0.3, 0.6))).to(dev)
+        for mode in ("dense", "sparse", "sparse_filter"):
+            cfg = dict(arch, attn_mode=synth.ATTN_DENSE if mode == "dense" else synth.ATTN_SPARSE, block=8, radius=1,
+                       filter_layer=4 if mode == "sparse_filter" else 0, keep_ratio=0.5 if mode == "sparse_filter" else 1.0)
+            wl = dict(name=f"vitl16_{side}_b{B}_{mode}", arch=arch, cfg=cfg, side=side, grid=g, batch=B)
+            torch.cuda.empty_cache()
+            torch.cuda.reset_peak_memory_stats()
+            steps = args.steps if side <= 2048 else max(1, args.steps // 3)
+            kept = None
+            for _ in range(2 if side <= 2048 else 1):
+                _, kept = ctx.vit_forward(cfg, dw, img, g, g)
+            ctx.check()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(steps):
+                ctx.vit_forward(cfg, dw, img, g, g)
+            e1.record()
+            torch.cuda.synchronize()
+            ctx.check()
+            ms = e0.elapsed_time(e1) / steps
+            fl = forward_flops(dict(wl, cfg=dict(cfg, radius=g if mode == "dense" else 1)),
+                               None if kept is None else kept.cpu().numpy())
+            useful = fl["gemm"] + fl["attn_patch"] + fl["attn_global"]
+            print(json.dumps({"workload": wl["name"], "image": f"{side}x{side}", "tokens": 1 + g * g, "mode": mode,
+                              "batch": B, "ms_per_step": ms, "images_per_s": B / (ms * 1e-3),
+                              "useful_tflops": useful / (ms * 1e-3) / 1e12,
+                              "frac_of_bf16_peak": useful / (ms * 1e-3) / 1e12 / pk["tensor"],
+                              "attention_density": fl["attn_patch"] / max(1.0, forward_flops(
+                                  dict(wl, cfg=dict(cfg, radius=g, filter_layer=0)), None)["attn_patch"]),
+                              "peak_hbm_bytes": torch.cuda.max_memory_allocated(), "steps": steps}), flush=True)
+        del dw, img
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -472,7 +526,13 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--quick", action="store_true",
                     help="profiling aid: exactly --warmup warm-up steps, no end-to-end and no CPU leg")
+    ap.add_argument("--sweep", action="store_true",
+                    help="resolution sweep (dense / sparse / sparse+filter), one JSON line per point")
+    ap.add_argument("--sweep-sides", default="224,448,1024,2048,3072,4096")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     wl = workload_config(args.workload)
