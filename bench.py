@@ -191,7 +191,7 @@ def oracle_sample(wl, rows, seed=11):
     fl = c["filter_layer"]
     k = oracle.keep_count(np0, c["keep_ratio"]) if fl > 0 else np0
     n1 = G + k
-    rows = min(rows, n1)
+    rows = min(rows, n0)
     x = rng.standard_normal((rows, D), dtype=np.float32)
     cols = synth.round_bf16(rng.standard_normal((rows, 3 * a["patch"] ** 2), dtype=np.float32))
     t = {}
@@ -217,7 +217,7 @@ def oracle_sample(wl, rows, seed=11):
 
     def attn(n_tok, positions):
         q, kk, v = synth.attention_qkv(seed + n_tok, 1, n_tok, H, D // H)
-        qrows = np.sort(rng.choice(n_tok, size=rows, replace=False)).astype(np.int32)
+        qrows = np.sort(rng.choice(n_tok, size=rows, replace=rows > n_tok)).astype(np.int32)
         pp = None if positions is None else positions[None].astype(np.int32)
         t0 = time.perf_counter()
         oracle.attention(q, kk, v, g, g, c["block"], c["radius"], n_global=G, patch_pos=pp, rows=qrows)
