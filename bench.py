@@ -37,6 +37,8 @@ WORKLOADS = {
     "vitl16_1024_b1_sparse_filter": ("l16", 1024, 1, 8, 1, 4, 0.6, 2, 3),
     "vitl16_1024_b4_sparse_filter": ("l16", 1024, 4, 8, 1, 4, 0.5, 2, 6),
     "vitl16_448_b4_sparse_filter": ("l16", 448, 4, 8, 1, 4, 0.5, 2, 6),
+    # ViT-g/14-style: 40 layers, d 1536, 24 heads, SwiGLU 4096; 146x146 grid, 5x5 block neighbourhood
+    "vitg14_2044_b1_sparse_filter": ("g14", 2044, 1, 8, 2, 8, 0.5, 4, 5),
 }
 DEFAULT_WORKLOAD = "vitl16_2048_b4_sparse_filter"
 
