@@ -67,6 +67,9 @@ def test_single_attention_op_28x28(ctx):
     (12, 12, 2, 1, 1, 1, 2),      # small blocks: many blocks per query tile
     (20, 20, 16, 0, 1, 1, 2),     # blocks larger than a tile (256 tokens), own block only
     (9, 30, 4, 3, 1, 2, 1),       # wide neighbourhood
+    (12, 12, 1, 1, 1, 1, 2),      # one patch per block: 3x3-patch windows, a query tile per grid row
+    (10, 14, 3, 0, 8, 1, 1),      # own block only, the maximum of eight global tokens
+    (5, 3, 8, 1, 1, 1, 1),        # a grid smaller than one block
 ])
 def test_geometries(ctx, gh, gw, b, r, G, B, H):
     n = G + gh * gw
@@ -176,3 +179,16 @@ def test_sampled_rows_filtered_full_size(ctx):
     rows = np.unique(np.concatenate([[0, 1, 8192], rng.integers(1, 8193, size=250)])).astype(np.int32)
     want, _ = oracle.attention(q, k, v, gh, gw, 8, 1, patch_pos=pos_bm, rows=rows)
     _check(got[:, rows], want[:, rows])
+
+
+def test_blocks_larger_than_many_tiles(ctx):
+    """64x64-patch blocks (the largest window of the paper's ablation): 4096 tokens per block, 32 query
+    tiles per block, radius 0 and radius 1 on a 64x192 grid (1x3 blocks); sampled rows."""
+    gh, gw = 64, 192
+    q, k, v = synth.attention_qkv(6, 1, 1 + gh * gw, 1, 64)
+    rng = np.random.default_rng(3)
+    rows = np.unique(np.concatenate([[0, 1, gh * gw], rng.integers(1, 1 + gh * gw, size=120)])).astype(np.int32)
+    for r in (0, 1):
+        got, _ = _run(ctx, q, k, v, gh, gw, 64, r, scores=False)
+        want, _ = oracle.attention(q, k, v, gh, gw, 64, r, rows=rows)
+        _check(got[:, rows], want[:, rows])
