@@ -238,7 +238,10 @@ enum {
   SPV_EPI_BIAS_ADDROW = 5  /* resid fp32 [M, N] = acc + bias + addrow[(m % rows_per_image)]  */
 };
 
-/* C[M, N] = A[M, K] * W[N, K]^T (+ epilogue).  a, w: bf16 device, row-major with leading
+/* The residual epilogue adds into `out` with fp32 add-reduce operations issued by the kernel (each
+ * element receives exactly one add per call, so the result is deterministic); `out` must not be
+ * read or written by other work on the GPU while the call runs.
+ * C[M, N] = A[M, K] * W[N, K]^T (+ epilogue).  a, w: bf16 device, row-major with leading
  * dimensions lda, ldw (elements, multiples of 8); K multiple of 8.  out: bf16 [M, ldo] for the
  * bf16 epilogues, fp32 residual [M, ldo] for the residual ones.  bias fp32 [N] or NULL. */
 typedef struct {
