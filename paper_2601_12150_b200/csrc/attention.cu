@@ -586,92 +586,116 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 // ------------------------------------------------------------------------------------------
 // global-query rows
 // ------------------------------------------------------------------------------------------
-constexpr int GCH = 512;   // keys per CTA
+constexpr int GCH = 512;   // fewest keys per CTA (bounds the number of chunk partials)
 
-// grid (chunks, heads, batch * G).  Writes scaled logits, and per chunk (max, sum, sum p*v).
-__global__ void __launch_bounds__(256) attn_global_partial(const __nv_bfloat16* __restrict__ q,
+// grid (heads, chunks, batch * G).  One pass over the chunk's keys: every group of eight lanes walks
+// keys k0 + grp, k0 + grp + 32, ... with its own running (max, sum, sum p*v) -- the key and the value
+// row of a key are loaded together, so twice as many loads are in flight as with a score pass
+// followed by a value pass -- and the 32 group states are merged through shared memory.  Writes the
+// chunk's (max, sum, sum p*v) and, when the scores are wanted, the scaled logits.
+template <bool kLogits>
+__global__ void __launch_bounds__(256, 3) attn_global_partial(const __nv_bfloat16* __restrict__ q,
                                                            const __nv_bfloat16* __restrict__ k,
                                                            const __nv_bfloat16* __restrict__ v, int64_t sb,
                                                            int64_t st, int64_t sh, int n_tok, int n_global,
                                                            int heads, float scale, float* __restrict__ logits,
                                                            float* __restrict__ part_ml, float* __restrict__ part_o,
-                                                           int n_chunks) {
-  __shared__ float s_s[GCH];
-  __shared__ float s_red[32];
+                                                           int n_chunks, int chunk_len) {
+  __shared__ float s_m[32], s_l[32];
   __shared__ float s_o[32][HD + 1];
   // heads fastest: the CTAs running together read whole token rows (all heads) of one key chunk
   const int h = blockIdx.x, chunk = blockIdx.y, bg = blockIdx.z;
   const int b = bg / n_global, g = bg % n_global;
-  const int k0 = chunk * GCH, k1 = min(k0 + GCH, n_tok);
+  const int k0 = chunk * chunk_len, k1 = min(k0 + chunk_len, n_tok);
   const int sub = threadIdx.x & 7, grp = threadIdx.x >> 3;   // 8 lanes per key, 32 keys in flight
   float qf[8];
   unpack8(__ldg(reinterpret_cast<const uint4*>(q + b * sb + (int64_t)g * st + (int64_t)h * sh) + sub), qf);
-  for (int i = threadIdx.x; i < GCH; i += 256) s_s[i] = -INFINITY;
-  __syncthreads();
-  float lmax = -INFINITY;
-  // the trip count is the same for every lane (the shuffles name the whole warp); keys past the
-  // end of the chunk are predicated off
-#pragma unroll 4
-  for (int kk0 = k0; kk0 < k1; kk0 += 32) {
-    const int kk = kk0 + grp;
-    const bool live = kk < k1;
-    float d = 0.f;
-    if (live) {
-      float kf[8];
-      unpack8(__ldg(reinterpret_cast<const uint4*>(k + b * sb + (int64_t)kk * st + (int64_t)h * sh) + sub), kf);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) d = fmaf(qf[i], kf[i], d);
-    }
-    d += __shfl_xor_sync(0xffffffffu, d, 1);
-    d += __shfl_xor_sync(0xffffffffu, d, 2);
-    d += __shfl_xor_sync(0xffffffffu, d, 4);
-    d *= scale;
-    if (live) {
-      if (sub == 0) s_s[kk - k0] = d;
-      lmax = fmaxf(lmax, d);
-    }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) lmax = fmaxf(lmax, __shfl_xor_sync(0xffffffffu, lmax, o));
-  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = lmax;
-  __syncthreads();
-  float cmax = s_red[0];
-#pragma unroll
-  for (int w = 1; w < 8; ++w) cmax = fmaxf(cmax, s_red[w]);
   float* lg = logits + ((size_t)bg * heads + h) * n_tok;
-  float lsum = 0.f;
-  for (int i = threadIdx.x; i < k1 - k0; i += 256) {
-    const float s = s_s[i];
-    lg[k0 + i] = s;
-    lsum += __expf(s - cmax);
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) s_red[8 + (threadIdx.x >> 5)] = lsum;
+  float m = -INFINITY, l = 0.f;
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll 4
-  for (int kk = k0 + grp; kk < k1; kk += 32) {
-    const float pw = __expf(s_s[kk - k0] - cmax);
-    float vf[8];
-    unpack8(__ldg(reinterpret_cast<const uint4*>(v + b * sb + (int64_t)kk * st + (int64_t)h * sh) + sub), vf);
+  // the trip count is the same for every lane (the shuffles name the whole warp); keys past the
+  // end of the chunk are predicated off.  The loads of GU keys (key and value rows) are issued
+  // before any of them is used.
+  constexpr int GU = 4;
+#pragma unroll 1
+  for (int kk0 = k0; kk0 < k1; kk0 += 32 * GU) {
+    uint4 ku[GU], vu[GU];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] = fmaf(pw, vf[i], acc[i]);
+    for (int u = 0; u < GU; ++u) {
+      const int kk = kk0 + u * 32 + grp;
+      ku[u] = make_uint4(0u, 0u, 0u, 0u);
+      vu[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (kk < k1) {
+        const int64_t off = b * sb + (int64_t)kk * st + (int64_t)h * sh;
+        ku[u] = __ldg(reinterpret_cast<const uint4*>(k + off) + sub);
+        vu[u] = __ldg(reinterpret_cast<const uint4*>(v + off) + sub);
+      }
+    }
+    float d[GU];
+#pragma unroll
+    for (int u = 0; u < GU; ++u) {
+      float kf[8];
+      unpack8(ku[u], kf);
+      d[u] = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) d[u] = fmaf(qf[i], kf[i], d[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < GU; ++u) {
+      d[u] += __shfl_xor_sync(0xffffffffu, d[u], 1);
+      d[u] += __shfl_xor_sync(0xffffffffu, d[u], 2);
+      d[u] += __shfl_xor_sync(0xffffffffu, d[u], 4);
+      d[u] = (kk0 + u * 32 + grp < k1) ? d[u] * scale : -INFINITY;
+    }
+    if (kLogits && sub < GU) {
+      // lane u of the group writes key u's logit
+      float mine = d[0];
+#pragma unroll
+      for (int u = 1; u < GU; ++u) mine = sub == u ? d[u] : mine;
+      const int kk = kk0 + sub * 32 + grp;
+      if (kk < k1) lg[kk] = mine;
+    }
+    float mx = d[0];
+#pragma unroll
+    for (int u = 1; u < GU; ++u) mx = fmaxf(mx, d[u]);
+    if (mx > m) {                        // the same decision in all eight lanes of the group
+      const float a = __expf(m - mx);    // m = -inf on the first batch: a = 0, the state is empty
+      l *= a;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] *= a;
+      m = mx;
+    }
+    const float mref = m == -INFINITY ? 0.f : m;   // a group that has seen no key yet: every p below is 0
+#pragma unroll
+    for (int u = 0; u < GU; ++u) {
+      const float pw = __expf(d[u] - mref);          // 0 for a key past the end of the chunk
+      float vf[8];
+      unpack8(vu[u], vf);
+      l += pw;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] = fmaf(pw, vf[i], acc[i]);
+    }
   }
+  if (sub == 0) { s_m[grp] = m; s_l[grp] = l; }
 #pragma unroll
   for (int i = 0; i < 8; ++i) s_o[grp][sub * 8 + i] = acc[i];
   __syncthreads();
+  float cmax = -INFINITY;
+#pragma unroll
+  for (int gI = 0; gI < 32; ++gI) cmax = fmaxf(cmax, s_m[gI]);
   const size_t pidx = ((size_t)bg * heads + h) * n_chunks + chunk;
   if (threadIdx.x < HD) {
     float t = 0.f;
 #pragma unroll
-    for (int gI = 0; gI < 32; ++gI) t += s_o[gI][threadIdx.x];
+    for (int gI = 0; gI < 32; ++gI)
+      if (s_m[gI] > -INFINITY) t += s_o[gI][threadIdx.x] * __expf(s_m[gI] - cmax);
     part_o[pidx * HD + threadIdx.x] = t;
   }
   if (threadIdx.x == 0) {
     float t = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) t += s_red[8 + w];
+    for (int gI = 0; gI < 32; ++gI)
+      if (s_m[gI] > -INFINITY) t += s_l[gI] * __expf(s_m[gI] - cmax);
     part_ml[pidx * 2] = cmax;
     part_ml[pidx * 2 + 1] = t;
   }
@@ -845,15 +869,23 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   const int n_tok = plan->n_global + plan->n_patch, G = plan->n_global, B = plan->batch;
   if (ws_bytes < spv_attn_global_bytes(B, G, io->heads, n_tok)) return SPV_ERR_WORKSPACE;
   const size_t rows = (size_t)B * G * io->heads;
-  const int chunks = (n_tok + GCH - 1) / GCH;
+  // as many chunks as fill the GPU once (three CTAs of this kernel per SM), none shorter than GCH keys
+  const int max_chunks = (n_tok + GCH - 1) / GCH;
+  int chunks = (int)((size_t)ctx->sm_count * 3 / rows);
+  chunks = chunks < 1 ? 1 : (chunks > max_chunks ? max_chunks : chunks);
+  const int chunk_len = ((n_tok + chunks - 1) / chunks + 127) / 128 * 128;
+  chunks = (n_tok + chunk_len - 1) / chunk_len;
   char* w = (char*)ws;
   float* logits = (float*)w; w += spv_align_up(rows * n_tok * 4, 256);
   float* part_ml = (float*)w; w += spv_align_up(rows * chunks * 2 * 4, 256);
   float* part_o = (float*)w;
   SpvProfScope prof(ctx, SPV_K_ATTN_GLOBAL, stream);
-  attn_global_partial<<<dim3(io->heads, chunks, B * G), 256, 0, stream>>>(
+  if (scores) attn_global_partial<true><<<dim3(io->heads, chunks, B * G), 256, 0, stream>>>(
       (const __nv_bfloat16*)io->q, (const __nv_bfloat16*)io->k, (const __nv_bfloat16*)io->v, io->sb, io->st, io->sh,
-      n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks);
+      n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks, chunk_len);
+  else attn_global_partial<false><<<dim3(io->heads, chunks, B * G), 256, 0, stream>>>(
+      (const __nv_bfloat16*)io->q, (const __nv_bfloat16*)io->k, (const __nv_bfloat16*)io->v, io->sb, io->st, io->sh,
+      n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks, chunk_len);
   attn_global_combine<<<dim3(io->heads, B * G), 256, 0, stream>>>(logits, part_ml, part_o, chunks, n_tok, G,
                                                                  io->heads, (__nv_bfloat16*)io->o, io->o_sb,
                                                                  io->o_st, io->o_sh, scores, score_idx);
