@@ -38,22 +38,37 @@ struct EpiParams {
 // (|error| <= 1.5e-7, branch-free: one reciprocal, one exponential, five multiply-adds), which keeps
 // the epilogue of the MLP GEMM shorter than its main loop; the absolute error of the GELU value is
 // below |x| * 1e-7, far inside the bf16 rounding of the stored activation.
-__device__ __forceinline__ float gelu_erf(float x) {
-  const float z = fabsf(x) * 0.70710678118654752f;
-  float t;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, z, 1.0f)));
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  poly *= t;
-  float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(z * z * -1.4426950408889634f));
-  const float erf_abs = fmaf(-poly, e, 1.0f);           // erf(|x| / sqrt 2)
-  const float half_x = 0.5f * x;
-  return fmaf(fabsf(half_x), erf_abs, half_x);          // 0.5 x (1 + sign(x) erf(|x|/sqrt 2))
+// Two values at a time: the multiply-adds run as packed fp32x2 instructions.
+__device__ __forceinline__ float2 gelu_erf2(float2 x) {
+  const float2 ax = make_float2(fabsf(x.x), fabsf(x.y));
+  const float2 z = __fmul2_rn(ax, make_float2(0.70710678118654752f, 0.70710678118654752f));
+  const float2 den = __ffma2_rn(make_float2(0.3275911f, 0.3275911f), z, make_float2(1.0f, 1.0f));
+  float2 t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.x) : "f"(den.x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.y) : "f"(den.y));
+  float2 poly = __ffma2_rn(make_float2(1.061405429f, 1.061405429f), t, make_float2(-1.453152027f, -1.453152027f));
+  poly = __ffma2_rn(poly, t, make_float2(1.421413741f, 1.421413741f));
+  poly = __ffma2_rn(poly, t, make_float2(-0.284496736f, -0.284496736f));
+  poly = __ffma2_rn(poly, t, make_float2(0.254829592f, 0.254829592f));
+  poly = __fmul2_rn(poly, t);
+  const float2 arg = __fmul2_rn(__fmul2_rn(z, z), make_float2(-1.4426950408889634f, -1.4426950408889634f));
+  float2 e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(arg.x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(arg.y));
+  const float2 neg_poly = make_float2(-poly.x, -poly.y);
+  const float2 erf_abs = __ffma2_rn(neg_poly, e, make_float2(1.0f, 1.0f));        // erf(|x| / sqrt 2)
+  const float2 half_x = __fmul2_rn(x, make_float2(0.5f, 0.5f));
+  // 0.5 x (1 + sign(x) erf(|x|/sqrt 2))
+  return __ffma2_rn(make_float2(fabsf(half_x.x), fabsf(half_x.y)), erf_abs, half_x);
 }
-__device__ __forceinline__ float silu(float x) { return x / (1.0f + __expf(-x)); }
+// x * sigmoid(x) with the hardware exponential and reciprocal (relative error about 1e-6, far
+// inside the bf16 rounding of the stored value); exp(-x) = inf for x < -88 gives 1/inf = 0, so x * 0 = -0
+__device__ __forceinline__ float silu(float x) {
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * -1.4426950408889634f));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+  return x * r;
+}
 
 __host__ __device__ constexpr bool epi_is_f32(int epi) { return epi == SPV_EPI_BIAS_SCALE_RESID || epi == SPV_EPI_BIAS_ADDROW; }
 
@@ -71,7 +86,11 @@ __device__ __forceinline__ void epilogue_math(const EpiParams& p, int m, int n, 
   }
   if constexpr (EPI == SPV_EPI_BIAS_GELU) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = gelu_erf(v[i]);
+    for (int i = 0; i < 8; i += 2) {
+      const float2 g = gelu_erf2(make_float2(v[i], v[i + 1]));
+      v[i] = g.x;
+      v[i + 1] = g.y;
+    }
   } else if constexpr (EPI == SPV_EPI_BIAS_SILU) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = silu(v[i]);
