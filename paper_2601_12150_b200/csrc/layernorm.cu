@@ -1,14 +1,18 @@
 // LayerNorm over fp32 residual rows, bf16 output (pre-LN of every ViT block and the final norm).
 // One warp per row, 128-bit loads, the row kept in registers between the statistics and the
-// normalisation, so each element crosses HBM once in (4 B) and once out (2 B).
+// normalisation, so each element crosses HBM once in (4 B) and once out (2 B).  The grid is
+// persistent (as many CTAs as are resident at once) and every warp issues the loads of its next
+// row before it reduces, normalises and stores the current one, so loads stay in flight the
+// whole time.
 #include "common.cuh"
 
 namespace {
 
-// kMaxVec float4 per lane are held in registers (dim <= 128 * kMaxVec); the instantiation that just
-// covers the row keeps the register count low, so that more warps (more loads in flight) fit an SM.
+// kMaxVec float4 per lane are held in registers for the current row and as many for the next one
+// (dim <= 128 * kMaxVec); the instantiation that just covers the row keeps the register count low,
+// so that two CTAs fit an SM up to dim 1024.
 template <int kMaxVec>
-__global__ void __launch_bounds__(256, (kMaxVec <= 8 ? 3 : 2)) layernorm_kernel(const float* __restrict__ x, int64_t rows, int dim,
+__global__ void __launch_bounds__(256, (kMaxVec <= 8 ? 2 : 1)) layernorm_kernel(const float* __restrict__ x, int64_t rows, int dim,
                                                         const float* __restrict__ gamma,
                                                         const float* __restrict__ beta, float eps,
                                                         __nv_bfloat16* __restrict__ y,
@@ -18,6 +22,15 @@ __global__ void __launch_bounds__(256, (kMaxVec <= 8 ? 3 : 2)) layernorm_kernel(
   const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
   const int nvec = dim >> 2;
   const float inv_dim = 1.0f / (float)dim;
+  float4 nxt[kMaxVec];          // the row after the current one, in flight
+  if (warp < rows) {
+    const float4* xr0 = reinterpret_cast<const float4*>(x + warp * dim);
+#pragma unroll
+    for (int i = 0; i < kMaxVec; ++i) {
+      const int c = lane + 32 * i;
+      if (c < nvec) nxt[i] = __ldcs(xr0 + c);
+    }
+  }
   for (int64_t r = warp; r < rows; r += nwarps) {
     const float4* xr = reinterpret_cast<const float4*>(x + r * dim);
     float4 v[kMaxVec];
@@ -26,8 +39,16 @@ __global__ void __launch_bounds__(256, (kMaxVec <= 8 ? 3 : 2)) layernorm_kernel(
     for (int i = 0; i < kMaxVec; ++i) {
       const int c = lane + 32 * i;
       if (c < nvec) {
-        v[i] = __ldcs(xr + c);
+        v[i] = nxt[i];
         sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+      }
+    }
+    if (r + nwarps < rows) {
+      const float4* xn = reinterpret_cast<const float4*>(x + (r + nwarps) * dim);
+#pragma unroll
+      for (int i = 0; i < kMaxVec; ++i) {
+        const int c = lane + 32 * i;
+        if (c < nvec) nxt[i] = __ldcs(xn + c);
       }
     }
     for (int c = lane + 32 * kMaxVec; c < nvec; c += 32) {
@@ -89,7 +110,7 @@ extern "C" int32_t spv_layernorm(spv_ctx* ctx, const float* x, int64_t rows, int
   if (((uintptr_t)x & 15u) || ((uintptr_t)y & 15u) || ((uintptr_t)gamma & 15u) || ((uintptr_t)beta & 15u))
     return SPV_ERR_ALIGNMENT;
   int64_t blocks = (rows + 7) / 8;
-  const int64_t cap = (int64_t)ctx->sm_count * 64;
+  const int64_t cap = (int64_t)ctx->sm_count * (dim <= 1024 ? 2 : 1);     // resident CTAs (see __launch_bounds__)
   if (blocks > cap) blocks = cap;
   SpvProfScope prof(ctx, SPV_K_LAYERNORM, (cudaStream_t)stream, (double)rows * dim * 6.0);
   const unsigned g = (unsigned)blocks;
