@@ -1,8 +1,14 @@
 // bf16 GEMM with fused epilogues for the ViT block (QKV / out-proj / MLP / patch embedding):
 //   C[M, N] = A[M, K] * W[N, K]^T, fp32 accumulation in TMEM.
 //
-// Persistent kernel, one CTA per SM, 128 x 256 output tiles, K in slices of 64:
-//   warp 0      TMA producer (A and W slices, 128-byte swizzle, 4-stage ring)
+// Persistent kernel, one CTA per SM, K in slices of 64.  Two forms of the same body:
+//   pair form   (M > 256) two CTAs of a cluster share one tcgen05.mma.cta_group::2 of shape
+//               256 x 256 x 16: each CTA loads 128 rows of A and 128 of the 256 rows of W, the
+//               even CTA issues the MMAs, each CTA's TMEM gets its 128 x 256 half of the tile and
+//               each CTA runs its own epilogue.  A W slice crosses L2 -> shared memory once per
+//               256 output rows instead of once per 128, and a stage is 32 KB (6-stage ring).
+//   single form 128 x 256 tiles, 48 KB stages (4-stage ring), for small M.
+//   warp 0      TMA producer (A and W slices, 128-byte swizzle)
 //   warp 1      tcgen05.mma issuer (one thread), owns the TMEM allocation (2 x 256 columns, so
 //               the epilogue of tile i overlaps the main loop of tile i+1)
 //   warps 2..9  epilogue, two threads per output row: TMEM -> registers -> bias / activation /
@@ -15,12 +21,17 @@ namespace {
 
 using namespace spv;
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int A_BYTES = BM * BK * 2;
+template <bool PAIR> struct Ring {
+  static constexpr int STAGES = PAIR ? 6 : 4;
+  static constexpr int B_ROWS = PAIR ? BN / 2 : BN;       // rows of W one CTA loads per slice
+  static constexpr int B_BYTES = B_ROWS * BK * 2;
+};
 constexpr int GEMM_THREADS = 320;      // warp 0 TMA, warp 1 MMA, warps 2-9 epilogue (two per TMEM lane quadrant)
 constexpr int EPI_THREADS = 256;
 constexpr int EPI_BYTES = 128 * 128;    // one staging buffer: 128 rows x 128 bytes (32 fp32 or 64 bf16 columns)
-constexpr int GEMM_SMEM = STAGES * (A_BYTES + B_BYTES) + 2 * EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int GEMM_SMEM = 4 * (A_BYTES + BN * BK * 2) + 2 * EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/;   // both forms: 192 KB of ring
 
 struct EpiParams {
   void* out;
@@ -120,12 +131,13 @@ __device__ __forceinline__ void epilogue_math(const EpiParams& p, int m, int n, 
   }
 }
 
-template <int EPI>
+template <int EPI, bool PAIR>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
                  const __grid_constant__ CUtensorMap tm_out, int M, int N, int K, EpiParams ep, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr int STAGES = Ring<PAIR>::STAGES, B_BYTES = Ring<PAIR>::B_BYTES;
   uint8_t* sA = smem;
   uint8_t* sB = smem + STAGES * A_BYTES;
   uint8_t* sE = smem + STAGES * (A_BYTES + B_BYTES);     // [2] epilogue staging, 128-byte swizzle
@@ -138,19 +150,27 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m_tiles = (M + BM - 1) / BM, n_tiles = (N + BN - 1) / BN;
+  // pair form: a tile is 256 rows, CTA `rank` of the pair owns rows [128 rank, 128 rank + 128) of it
+  // and loads rows [128 rank, 128 rank + 128) of the tile's 256 rows of W; the workers are the pairs
+  constexpr int TILE_M = PAIR ? 2 * BM : BM;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int m_tiles = (M + TILE_M - 1) / TILE_M, n_tiles = (N + BN - 1) / BN;
   const int tiles = m_tiles * n_tiles;
   const int kblocks = (K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], EPI_THREADS); }
+    // pair form: the even CTA's MMA thread waits for the epilogues of both CTAs
+    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], PAIR ? 2 * EPI_THREADS : EPI_THREADS); }
     *abort_flag = 0;
     mbar_fence_init();
   }
+  if constexpr (PAIR) cluster_sync_all();      // both CTAs' barriers exist before anything remote touches them
   if (warp == 1) {
-    tmem_alloc(tmem_slot, 512);
-    tmem_relinquish();
+    if constexpr (PAIR) { tmem_alloc_pair(tmem_slot, 512); tmem_relinquish_pair(); }
+    else { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
   }
   tc_fence_before();
   __syncthreads();
@@ -162,24 +182,32 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       tma_prefetch_desc(&tm_a);
       tma_prefetch_desc(&tm_w);
       uint32_t it = 0;
-      for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+      for (int tile = worker; tile < tiles; tile += n_workers) {
         // column tile fastest: the CTAs running together share a few row tiles of A and all of W in L2,
         // so A crosses HBM once instead of once per column tile
-        const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+        const int m0 = (tile / n_tiles) * TILE_M + (int)rank * BM, n0 = (tile % n_tiles) * BN;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % STAGES;
           mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, status, 0x100 + s);
-          mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
-          tma_load_2d(sA + s * A_BYTES, &tm_a, &full[s], kb * BK, m0);
-          tma_load_2d(sB + s * B_BYTES, &tm_w, &full[s], kb * BK, n0);
+          if constexpr (PAIR) {
+            // the bytes of both CTAs are counted on the even CTA's barrier, which its producer arms
+            if (rank == 0) mbar_expect_tx(&full[s], 2 * (A_BYTES + B_BYTES));
+            const uint32_t bar = mapa_shared(smem_u32(&full[s]), 0);
+            tma_load_2d_pair(sA + s * A_BYTES, &tm_a, bar, kb * BK, m0);
+            tma_load_2d_pair(sB + s * B_BYTES, &tm_w, bar, kb * BK, n0 + (int)rank * (BN / 2));
+          } else {
+            mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
+            tma_load_2d(sA + s * A_BYTES, &tm_a, &full[s], kb * BK, m0);
+            tma_load_2d(sB + s * B_BYTES, &tm_w, &full[s], kb * BK, n0);
+          }
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(BM, BN, false);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = idesc_bf16(TILE_M, BN, false);
       uint32_t it = 0, tcount = 0;
-      for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
+      for (int tile = worker; tile < tiles; tile += n_workers, ++tcount) {
         const int a = tcount & 1;
         mbar_wait(&acc_empty[a], ((tcount >> 1) & 1) ^ 1, abort_flag, status, 0x200 + a);
         tc_fence_after();
@@ -191,11 +219,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           const uint64_t da = smem_desc_sw128(smem_u32(sA + s * A_BYTES));
           const uint64_t db = smem_desc_sw128(smem_u32(sB + s * B_BYTES));
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)
-            mma_ss(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
-          tc_commit(&empty[s]);
+          for (int k = 0; k < BK / 16; ++k) {
+            if constexpr (PAIR) mma_ss_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+            else mma_ss(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+          }
+          if constexpr (PAIR) tc_commit_pair(&empty[s], 3);      // frees the stage in both CTAs
+          else tc_commit(&empty[s]);
         }
-        tc_commit(&acc_full[a]);
+        if constexpr (PAIR) tc_commit_pair(&acc_full[a], 3);     // both CTAs' epilogues may read their half
+        else tc_commit(&acc_full[a]);
       }
     }
   } else {
@@ -211,9 +243,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     const int row = q * 32 + lane;
     const bool issuer = threadIdx.x == 64;
     uint32_t tcount = 0, ec = 0;
-    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tcount) {
+    const uint32_t acc_empty_remote = PAIR ? mapa_shared(smem_u32(&acc_empty[0]), 0) : 0u;
+    for (int tile = worker; tile < tiles; tile += n_workers, ++tcount) {
       const int a = tcount & 1;
-      const int m_base = (tile / n_tiles) * BM, n_base = (tile % n_tiles) * BN;
+      const int m_base = (tile / n_tiles) * TILE_M + (int)rank * BM, n_base = (tile % n_tiles) * BN;
       const int m = m_base + row;
       mbar_wait(&acc_full[a], (tcount >> 1) & 1, abort_flag, status, 0x400 + a);
       tc_fence_after();
@@ -252,22 +285,30 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         }
         fence_async_smem();
         asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (issuer) {
+        if (issuer && m_base < M) {          // (the odd CTA's half of the last row tile may lie past M)
           if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID) tma_reduce_add_2d(&tm_out, buf, n0, m_base);
           else tma_store_2d(&tm_out, buf, n0, m_base);
           bulk_commit();
         }
       }
       tc_fence_before();
-      mbar_arrive(&acc_empty[a]);
+      if constexpr (PAIR) mbar_arrive_cluster(acc_empty_remote + 8u * (uint32_t)a);
+      else mbar_arrive(&acc_empty[a]);
     }
     if (issuer) bulk_wait<0>();
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();      // neither CTA frees TMEM or leaves while the other may still signal it
   tc_fence_after();
-  if (warp == 1) tmem_dealloc(tmem_base, 512);
+  if (warp == 1) {
+    if constexpr (PAIR) tmem_dealloc_pair(tmem_base, 512);
+    else tmem_dealloc(tmem_base, 512);
+  }
 }
+
+// the pair form pays off once a problem has more than one 256-row tile
+inline bool use_pair(const spv_gemm_desc* d) { return d->m > 2 * BM; }
 
 template <int EPI>
 int32_t launch(spv_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tw, const spv_gemm_desc* d, const EpiParams& ep,
@@ -287,15 +328,41 @@ int32_t launch(spv_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tw, const
     }
     if (st != SPV_OK) return st;
   }
+  SpvProfScope prof(ctx, SPV_K_GEMM, stream, 2.0 * (double)d->m * (double)d->n * (double)d->k);
+  const int n_tiles = (d->n + BN - 1) / BN;
+  if (use_pair(d)) {
+    // pair form: clusters of two CTAs, as many as can be resident at once
+    static int max_pairs = 0;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = GEMM_SMEM;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (max_pairs == 0) {
+      SPV_CUDA_OK(cudaFuncSetAttribute(gemm_bf16_kernel<EPI, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
+      cfg.gridDim = dim3(2 * (ctx->sm_count / 2));
+      int n = 0;
+      SPV_CUDA_OK(cudaOccupancyMaxActiveClusters(&n, gemm_bf16_kernel<EPI, true>, &cfg));
+      if (n < 1) return SPV_ERR_CUDA;
+      max_pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
+    }
+    const int tiles = ((d->m + 2 * BM - 1) / (2 * BM)) * n_tiles;
+    cfg.gridDim = dim3(2 * (tiles < max_pairs ? tiles : max_pairs));
+    SPV_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_bf16_kernel<EPI, true>, ta, tw, tout, d->m, d->n, d->k, ep, ctx->d_status));
+    return spv_launch_ok(ctx);
+  }
   static bool configured = false;
   if (!configured) {
-    SPV_CUDA_OK(cudaFuncSetAttribute(gemm_bf16_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
+    SPV_CUDA_OK(cudaFuncSetAttribute(gemm_bf16_kernel<EPI, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
     configured = true;
   }
-  const int tiles = ((d->m + BM - 1) / BM) * ((d->n + BN - 1) / BN);
+  const int tiles = ((d->m + BM - 1) / BM) * n_tiles;
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-  SpvProfScope prof(ctx, SPV_K_GEMM, stream, 2.0 * (double)d->m * (double)d->n * (double)d->k);
-  gemm_bf16_kernel<EPI><<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tw, tout, d->m, d->n, d->k, ep, ctx->d_status);
+  gemm_bf16_kernel<EPI, false><<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tw, tout, d->m, d->n, d->k, ep, ctx->d_status);
   return spv_launch_ok(ctx);
 }
 
@@ -326,7 +393,7 @@ extern "C" int32_t spv_gemm_bf16(spv_ctx* ctx, const spv_gemm_desc* d, const voi
   {
     const uint64_t dims[2] = {(uint64_t)d->k, (uint64_t)d->n};
     const uint64_t str[1] = {(uint64_t)d->ldw * 2};
-    const uint32_t box[2] = {BK, BN};
+    const uint32_t box[2] = {BK, (uint32_t)(use_pair(d) ? BN / 2 : BN)};
     int32_t st = spv_make_tmap_bf16(ctx, &tw, w, 2, dims, str, box);
     if (st != SPV_OK) return st;
   }

@@ -29,8 +29,13 @@ def _check(got, ref, max_abs=2e-2, rel_l2=5e-3):
     assert np.linalg.norm(err) / max(np.linalg.norm(ref), 1e-30) <= rel_l2
 
 
+# M <= 256 runs on single CTAs with 128-row tiles, M > 256 on CTA pairs with 256-row tiles.  (257, ...)
+# and (385, ...): the odd CTA's half of the last tile lies wholly past M; (256, ...): the largest
+# single-CTA problem; (640, 136, ...): a column tile of which the odd CTA's rows of W lie past N;
+# (20000, 1288, ...): more tiles than CTA pairs, ragged in M and N, several passes over the ring.
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (300, 512, 192), (1000, 264, 328), (77, 64, 1024),
-                                   (4097, 1024, 1024)])
+                                   (4097, 1024, 1024), (257, 256, 128), (385, 512, 64), (256, 512, 200),
+                                   (640, 136, 72), (20000, 1288, 456)])
 def test_gemm_fp32_residual_epilogue(ctx, M, N, K):
     """resid += scale * (A W^T + bias): fp32 output, so any mis-addressed tile or k-slice shows."""
     import paper_2601_12150_b200 as spv
@@ -49,10 +54,11 @@ def test_gemm_fp32_residual_epilogue(ctx, M, N, K):
     assert np.abs(out.cpu().numpy() - ref).max() < 2e-4
 
 
+@pytest.mark.parametrize("M", [389, 200])          # CTA pairs / single CTAs
 @pytest.mark.parametrize("epi", ["bias", "gelu", "silu", "mul", "addrow"])
-def test_gemm_epilogues(ctx, epi):
+def test_gemm_epilogues(ctx, epi, M):
     import paper_2601_12150_b200 as spv
-    M, N, K = 389, 520, 136
+    N, K = 520, 136
     rng = np.random.default_rng(5)
     a = synth.round_bf16(rng.standard_normal((M, K), dtype=np.float32))
     w = synth.round_bf16(rng.standard_normal((N, K), dtype=np.float32) * 0.1)
