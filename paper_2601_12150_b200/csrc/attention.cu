@@ -14,8 +14,9 @@
 //   attn_regroup       row-major -> block-major copy of Q, K, V (only for row-major callers)
 //   attn_patch_kernel  flash-style tcgen05 kernel: S = Q K^T into TMEM, online softmax by 128
 //                      row-owning threads, P written back to TMEM as bf16, O += P V with V as an
-//                      MN-major shared-memory operand; global tokens enter as the initial
-//                      softmax state, so key tiles stay multiples of the MMA shape
+//                      MN-major shared-memory operand; the global tokens' keys and values join
+//                      the softmax state in the epilogue (dot products on the CUDA cores while
+//                      the last P V runs), so key tiles stay multiples of the MMA shape
 //   attn_global_*      the dense rows of the global (CLS) queries and the CLS->patch scores
 #include "attention.cuh"
 
@@ -367,34 +368,11 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int rlo = max(bxq - r, 0), rhi = min(bxq + r, p.nbx - 1);
     const float sl2 = p.scale_log2;
 
-    // global tokens: initial softmax state (m, l); their value rows are added in the epilogue
-    mbar_wait(q_full, 0, abort_flag, p.status, 0x1700);
-    float m = -INFINITY;
-    {
-      float qf[HD];
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const uint4 u = *reinterpret_cast<const uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4));
-        unpack8(u, qf + 8 * c);
-      }
-#pragma unroll 1
-      for (int g = 0; g < G; ++g) {
-        float d[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};     // eight independent chains
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          float kf[8];
-          unpack8(*reinterpret_cast<const uint4*>(sKg + g * 128 + ((c ^ (g & 7)) << 4)), kf);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) d[i] = fmaf(qf[8 * c + i], kf[i], d[i]);
-        }
-        const float sc = (((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]))) * sl2;
-        s_sg[g * 128 + row] = sc;
-        m = fmaxf(m, sc);
-      }
-    }
+    // The running maximum starts at a finite floor instead of -inf, so that a tile in which this
+    // row has no allowed key (all scores masked to -inf) gives p = 2^(-inf) = 0 and not 2^(nan).
+    // The global tokens join at the end (epilogue), while the last P V is still running.
+    float m = -1.0e30f;
     float l = 0.f;
-#pragma unroll 1
-    for (int g = 0; g < G; ++g) l += fast_exp2(s_sg[g * 128 + row] - m);
 
     uint32_t j = 0;
     for (int cy = cy0; cy <= cy1; ++cy) {
@@ -516,28 +494,63 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_arrive(p_full);
       }
     }
-    // ---------------- epilogue: O / l with the global tokens' share added
+    // ---------------- epilogue: the global tokens join the softmax, then O / l
+    // scaled scores of the global keys (their rows sit in shared memory since the Q tile arrived);
+    // computed before the wait for the last P V, which runs meanwhile
+    mbar_wait(q_full, 0, abort_flag, p.status, 0x1700);
+    float m_g = -INFINITY;
+    {
+      float qf[HD];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 u = *reinterpret_cast<const uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4));
+        unpack8(u, qf + 8 * c);
+      }
+#pragma unroll 1
+      for (int g = 0; g < G; ++g) {
+        float d[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};     // eight independent chains
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          float kf[8];
+          unpack8(*reinterpret_cast<const uint4*>(sKg + g * 128 + ((c ^ (g & 7)) << 4)), kf);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) d[i] = fmaf(qf[8 * c + i], kf[i], d[i]);
+        }
+        const float sc = (((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]))) * sl2;
+        s_sg[g * 128 + row] = sc;
+        m_g = fmaxf(m_g, sc);
+      }
+    }
+    const float m_f = fmaxf(m, m_g);                 // finite: there is at least one global key
+    const float a_p = fast_exp2(m - m_f);            // weight of everything accumulated so far
+    float l_f = l * a_p;
+#pragma unroll 1
+    for (int g = 0; g < G; ++g) l_f += fast_exp2(s_sg[g * 128 + row] - m_f);
+    const float inv = 1.0f / l_f;
     if (j > 0) {
       mbar_wait(pv_done, (j - 1) & 1, abort_flag, p.status, 0x1A00);
       tc_fence_after();
     }
     float of[HD];
+    {
+      const float a_o = a_p * inv;
 #pragma unroll
-    for (int c = 0; c < HD / 32; ++c) {
-      uint32_t orr[32];
-      if (j > 0) {
-        tmem_ld32(lane_addr + O_COL + 32 * c, orr);
-        tc_wait_ld();
-      } else {
+      for (int c = 0; c < HD / 32; ++c) {
+        uint32_t orr[32];
+        if (j > 0) {
+          tmem_ld32(lane_addr + O_COL + 32 * c, orr);
+          tc_wait_ld();
+        } else {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) orr[i] = 0u;
+          for (int i = 0; i < 32; ++i) orr[i] = 0u;
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) of[32 * c + i] = __uint_as_float(orr[i]) * a_o;
       }
-#pragma unroll
-      for (int i = 0; i < 32; ++i) of[32 * c + i] = __uint_as_float(orr[i]);
     }
 #pragma unroll 1
     for (int g = 0; g < G; ++g) {
-      const float w = fast_exp2(s_sg[g * 128 + row] - m);
+      const float w = fast_exp2(s_sg[g * 128 + row] - m_f) * inv;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         float vf[8];
@@ -549,14 +562,13 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // stage the bf16 row in the (now dead) Q tile, same 128-byte swizzle; each warp then stores its
     // own 32 rows, eight lanes per 128-byte row
     {
-      const float inv = 1.0f / l;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         uint4 w;
-        w.x = pack_bf16(of[8 * c] * inv, of[8 * c + 1] * inv);
-        w.y = pack_bf16(of[8 * c + 2] * inv, of[8 * c + 3] * inv);
-        w.z = pack_bf16(of[8 * c + 4] * inv, of[8 * c + 5] * inv);
-        w.w = pack_bf16(of[8 * c + 6] * inv, of[8 * c + 7] * inv);
+        w.x = pack_bf16(of[8 * c], of[8 * c + 1]);
+        w.y = pack_bf16(of[8 * c + 2], of[8 * c + 3]);
+        w.z = pack_bf16(of[8 * c + 4], of[8 * c + 5]);
+        w.w = pack_bf16(of[8 * c + 6], of[8 * c + 7]);
         *reinterpret_cast<uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4)) = w;
       }
     }
