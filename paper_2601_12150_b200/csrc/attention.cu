@@ -25,18 +25,21 @@ namespace {
 using namespace spv;
 
 constexpr int TQ = 128;            // query rows per tile (MMA M)
-constexpr int TK = 128;            // keys per tile (MMA N of S, K extent of P V)
+constexpr int TK = 64;             // keys per tile (MMA N of S, K extent of P V): with 64, a CTA needs 160 TMEM
+                                   // columns and 136 registers per softmax thread, so three CTAs fit an SM
 constexpr int HD = 64;             // head_dim
-constexpr int KST = 2;             // K / V smem stages
+constexpr int KST = 3;             // K / V smem stages
 constexpr int ATT_THREADS = 256;   // warps 0-3 softmax (one warpgroup), 4 TMA, 5 MMA, 6-7 idle: the second
                                    // warpgroup exists so that it can hand its registers to the first
-constexpr int TILE_BYTES = 128 * 128;
+constexpr int TILE_BYTES = 128 * 128;  // Q tile
+constexpr int KV_BYTES = TK * 128;      // K or V tile
 constexpr int GROW_BYTES = 1024;   // global-token rows of one head: up to 8 x 128 B
-constexpr int ATT_SMEM = TILE_BYTES * (1 + 2 * KST) + 2 * GROW_BYTES + 1024 /*align*/ + 256 /*barriers*/ +
+constexpr int ATT_SMEM = TILE_BYTES + 2 * KST * KV_BYTES + 2 * GROW_BYTES + 1024 /*align*/ + 256 /*barriers*/ +
                          8 * 128 * 4 /*global-token scores*/;
 constexpr int MAXG = 8;
-constexpr uint32_t TMEM_COLS = 256;
-constexpr uint32_t S_COL = 0, P_COL = 128, O_COL = 192;
+// two TMEM allocations per CTA, 160 columns in all, so that three CTAs share an SM's 512
+constexpr uint32_t TMEM_COLS = 128, TMEM_P_COLS = 32;
+constexpr uint32_t S_COL = 0, O_COL = 64;
 
 // ------------------------------------------------------------------------------------------
 // plan
@@ -230,7 +233,7 @@ __device__ __forceinline__ void unpack8(const uint4& u, float* f) {
   }
 }
 
-__global__ void __launch_bounds__(ATT_THREADS, 2)
+__global__ void __launch_bounds__(ATT_THREADS, 3)
 attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kg,
                   const __grid_constant__ CUtensorMap tm_vg, const PatchParams p) {
@@ -244,8 +247,8 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;
   uint8_t* sK = smem + TILE_BYTES;
-  uint8_t* sV = smem + TILE_BYTES * (1 + KST);
-  uint8_t* sKg = smem + TILE_BYTES * (1 + 2 * KST);      // global-token key rows (G x 128 B, swizzled)
+  uint8_t* sV = sK + KST * KV_BYTES;
+  uint8_t* sKg = sV + KST * KV_BYTES;      // global-token key rows (G x 128 B, swizzled)
   uint8_t* sVg = sKg + GROW_BYTES;                       // global-token value rows
   uint64_t* bars = reinterpret_cast<uint64_t*>(sVg + GROW_BYTES);
   uint64_t* q_full = bars;
@@ -282,17 +285,18 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   }
   if (warp == 5) {
     tmem_alloc(tmem_slot, TMEM_COLS);
+    tmem_alloc(tmem_slot + 2, TMEM_P_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem = *tmem_slot, tmem_p = tmem_slot[2];
 
-  // the softmax warpgroup holds a whole 128-column score row per thread; the other warpgroup
+  // the softmax warpgroup holds a whole score row of the key tile (64 columns) per thread; the other warpgroup
   // needs few registers
   if (warp >= 4) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 32;");
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 24;");
   if (warp == 4) {
     // ---------------- TMA producer
     if (lane == 0) {
@@ -308,11 +312,11 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           const int s = j % KST;
           const uint32_t ph = ((j / KST) & 1) ^ 1;
           mbar_wait(&k_empty[s], ph, abort_flag, p.status, 0x1100 + s);
-          mbar_expect_tx(&k_full[s], TILE_BYTES);
-          tma_load_4d(sK + s * TILE_BYTES, &tm_k, &k_full[s], 0, G + kb, h, b);
+          mbar_expect_tx(&k_full[s], KV_BYTES);
+          tma_load_4d(sK + s * KV_BYTES, &tm_k, &k_full[s], 0, G + kb, h, b);
           mbar_wait(&v_empty[s], ph, abort_flag, p.status, 0x1200 + s);
-          mbar_expect_tx(&v_full[s], TILE_BYTES);
-          tma_load_4d(sV + s * TILE_BYTES, &tm_v, &v_full[s], 0, G + kb, h, b);
+          mbar_expect_tx(&v_full[s], KV_BYTES);
+          tma_load_4d(sV + s * KV_BYTES, &tm_v, &v_full[s], 0, G + kb, h, b);
         }
       }
     }
@@ -332,7 +336,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_wait(&k_full[s], (j / KST) & 1, abort_flag, p.status, 0x1300 + s);
         if (j > 0) mbar_wait(s_free, (j - 1) & 1, abort_flag, p.status, 0x1400);
         tc_fence_after();
-        const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * TILE_BYTES));
+        const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * KV_BYTES));
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk)
           mma_ss(tmem + S_COL, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_s, kk != 0);
@@ -347,22 +351,23 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_wait(&v_full[s], (j / KST) & 1, abort_flag, p.status, 0x1500 + s);
         mbar_wait(p_full, j & 1, abort_flag, p.status, 0x1600);
         tc_fence_after();
-        const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * TILE_BYTES));
+        const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * KV_BYTES));
 #pragma unroll
         for (int kk = 0; kk < TK / 16; ++kk)
-          mma_ts(tmem + O_COL, tmem + P_COL + kk * 8, dv + (uint64_t)(kk * 128), idesc_o, (j | kk) != 0);
+          mma_ts(tmem + O_COL, tmem_p + kk * 8, dv + (uint64_t)(kk * 128), idesc_o, (j | kk) != 0);
         tc_commit(pv_done);
         tc_commit(&v_empty[s]);
       }
     }
   }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 136;");
     // ---------------- softmax + epilogue: thread `row` owns query row `row` (TMEM lane `row`)
     const int row = threadIdx.x;
     const int tok = q_begin + row;
     const bool valid = tok < q_end;
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_addr_p = tmem_p + ((uint32_t)(warp * 32) << 16);
     int bxq = bx_first;
     if (valid) bxq = __ldg(p.tok_blk + (size_t)b * p.n_patch + tok) % p.nbx;
     const int rlo = max(bxq - r, 0), rhi = min(bxq + r, p.nbx - 1);
@@ -485,7 +490,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
             for (int i = 0; i < 16; ++i) pk[i] = 0u;
           }
-          tmem_st16(lane_addr + P_COL + 16 * c, pk);
+          tmem_st16(lane_addr_p + 16 * c, pk);
         }
         l = l * alpha + ((rs_a.x + rs_a.y) + (rs_b.x + rs_b.y));
         m = m_new;
@@ -592,7 +597,10 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (warp == 5) tmem_dealloc(tmem, TMEM_COLS);
+  if (warp == 5) {
+    tmem_dealloc(tmem, TMEM_COLS);
+    tmem_dealloc(tmem_p, TMEM_P_COLS);
+  }
 }
 
 // ------------------------------------------------------------------------------------------
