@@ -402,24 +402,6 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const int i_hi = __reduce_min_sync(0xffffffffu, some ? c_hi : 0);
         mbar_wait(s_full, j & 1, abort_flag, p.status, 0x1800);
         tc_fence_after();
-        // boundary chunks (some of the warp's rows see only part of them) are masked in place
-        // first, by a small loop, so that the unrolled main pass below carries no mask code
-        // (none exist when every live chunk lies inside the intersection)
-        if (((u_lo & ~31) < i_lo) || (((u_hi + 31) & ~31) > i_hi)) {
-#pragma unroll 1
-        for (int cb = 0; cb < TK; cb += 32) {
-          if (cb < u_hi && cb + 32 > u_lo && !(cb >= i_lo && cb + 32 <= i_hi)) {
-            uint32_t t[32];
-            tmem_ld32(lane_addr + S_COL + cb, t);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (cb + i < c_lo || cb + i >= c_hi) t[i] = 0xff800000u;
-            tmem_st32(lane_addr + S_COL + cb, t);
-          }
-        }
-        tc_wait_st();
-        }
         // one pass: the live 32-column chunks of S go to registers, then S is released
         uint32_t sr[TK];
 #pragma unroll
@@ -428,6 +410,20 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tc_wait_ld();
         tc_fence_before();
         mbar_arrive(s_free);                               // S may be overwritten by the next Q K^T
+        // boundary chunks (some of the warp's rows see only part of them) are masked in registers:
+        // column c is allowed iff c_lo <= c < c_hi, one unsigned compare; chunks inside the
+        // intersection of the warp's rows skip this
+        {
+          const uint32_t width = (uint32_t)(c_hi - c_lo);
+#pragma unroll
+          for (int c = 0; c < TK / 32; ++c) {
+            if (32 * c < u_hi && 32 * c + 32 > u_lo && !(32 * c >= i_lo && 32 * c + 32 <= i_hi)) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if ((uint32_t)(32 * c + i - c_lo) >= width) sr[32 * c + i] = 0xff800000u;
+            }
+          }
+        }
         float mx = -INFINITY;
 #pragma unroll
         for (int c = 0; c < TK / 32; ++c) {
