@@ -602,7 +602,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 // ------------------------------------------------------------------------------------------
 // global-query rows
 // ------------------------------------------------------------------------------------------
-constexpr int GCH = 512;   // fewest keys per CTA (bounds the number of chunk partials)
+constexpr int GCH = 128;   // fewest keys per CTA (bounds the number of chunk partials)
 
 // grid (heads, chunks, batch * G).  One pass over the chunk's keys: every group of eight lanes walks
 // keys k0 + grp, k0 + grp + 32, ... with its own running (max, sum, sum p*v) -- the key and the value
