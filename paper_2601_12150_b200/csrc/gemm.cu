@@ -31,7 +31,7 @@ template <bool PAIR> struct Ring {
 constexpr int GEMM_THREADS = 320;      // warp 0 TMA, warp 1 MMA, warps 2-9 epilogue (two per TMEM lane quadrant)
 constexpr int EPI_THREADS = 256;
 constexpr int EPI_BYTES = 128 * 128;    // one staging buffer: 128 rows x 128 bytes (32 fp32 or 64 bf16 columns)
-constexpr int GEMM_SMEM = 4 * (A_BYTES + BN * BK * 2) + 2 * EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/;   // both forms: 192 KB of ring
+constexpr int GEMM_SMEM = 4 * (A_BYTES + BN * BK * 2) + 2 * EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/ + BN * 4 /*bias*/;   // both forms: 192 KB of ring
 
 struct EpiParams {
   void* out;
@@ -54,9 +54,11 @@ __device__ __forceinline__ float2 gelu_erf2(float2 x) {
   const float2 ax = make_float2(fabsf(x.x), fabsf(x.y));
   const float2 z = __fmul2_rn(ax, make_float2(0.70710678118654752f, 0.70710678118654752f));
   const float2 den = __ffma2_rn(make_float2(0.3275911f, 0.3275911f), z, make_float2(1.0f, 1.0f));
-  float2 t;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.x) : "f"(den.x));
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.y) : "f"(den.y));
+  // one reciprocal for the pair: 1/a = b / (a b), 1/b = a / (a b)  (a, b in [1, 1 + 0.23 |x|]); the
+  // special-function unit, at two operations per value, is what bounds this epilogue
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(den.x * den.y));
+  const float2 t = __fmul2_rn(make_float2(den.y, den.x), make_float2(r, r));
   float2 poly = __ffma2_rn(make_float2(1.061405429f, 1.061405429f), t, make_float2(-1.453152027f, -1.453152027f));
   poly = __ffma2_rn(poly, t, make_float2(1.421413741f, 1.421413741f));
   poly = __ffma2_rn(poly, t, make_float2(-0.284496736f, -0.284496736f));
@@ -86,12 +88,14 @@ __host__ __device__ constexpr bool epi_is_f32(int epi) { return epi == SPV_EPI_B
 // Eight consecutive outputs of row m, columns n .. n+7 (accumulators in acc), with the epilogue
 // arithmetic applied; the result stays fp32.
 template <int EPI>
-__device__ __forceinline__ void epilogue_math(const EpiParams& p, int m, int n, const uint32_t* acc, float* v) {
+__device__ __forceinline__ void epilogue_math(const EpiParams& p, const float* tile_bias, int n_base, int m, int n,
+                                              const uint32_t* acc, float* v) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(acc[i]);
   if (p.bias) {
-    const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + n));
-    const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + n + 4));
+    // the tile's 256 bias values sit in shared memory (tile_bias[0] belongs to column n_base)
+    const float4 b0 = *reinterpret_cast<const float4*>(tile_bias + (n - n_base));
+    const float4 b1 = *reinterpret_cast<const float4*>(tile_bias + (n - n_base) + 4);
     v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
     v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
   }
@@ -148,6 +152,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   uint64_t* acc_empty = bars + 2 * STAGES + 2;  // [2] epilogue -> MMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* s_bias = reinterpret_cast<float*>(bars + 32);     // [BN] bias of the tile in the epilogue
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // pair form: a tile is 256 rows, CTA `rank` of the pair owns rows [128 rank, 128 rank + 128) of it
@@ -248,6 +253,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       const int a = tcount & 1;
       const int m_base = (tile / n_tiles) * TILE_M + (int)rank * BM, n_base = (tile % n_tiles) * BN;
       const int m = m_base + row;
+      // the tile's bias goes to shared memory while the main loop still runs: a global load per
+      // chunk would sit (with its L2 latency) on the epilogue's critical path.  Every thread is past
+      // the last barrier of the previous tile here, so nobody still reads the old values; the
+      // first barrier of the chunk loop publishes the new ones.
+      if (ep.bias) {
+        const int tcol = threadIdx.x - 64;
+        s_bias[tcol] = n_base + tcol < N ? __ldg(ep.bias + n_base + tcol) : 0.f;
+      }
       mbar_wait(&acc_full[a], (tcount >> 1) & 1, abort_flag, status, 0x400 + a);
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
@@ -267,7 +280,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           float v[8];
           const int n = n0 + half * TW + 8 * g;
           if (m < M && n < N) {
-            epilogue_math<EPI>(ep, m, n, acc + 8 * g, v);
+            epilogue_math<EPI>(ep, s_bias, n_base, m, n, acc + 8 * g, v);
           } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = 0.f;
