@@ -11,7 +11,7 @@
 //   warp 0      TMA producer (A and W slices, 128-byte swizzle)
 //   warp 1      tcgen05.mma issuer (one thread), owns the TMEM allocation (2 x 256 columns, so
 //               the epilogue of tile i overlaps the main loop of tile i+1)
-//   warps 2..9  epilogue, two threads per output row: TMEM -> registers -> bias / activation /
+//   warps 2..17 epilogue, four threads per output row: TMEM -> registers -> bias / activation /
 //               scale -> swizzled staging buffer -> TMA tile store (bf16 outputs, fp32 rows) or
 //               fp32 TMA add-reduce into the residual stream
 // Rows beyond M and columns beyond N are zero-filled by TMA on load and clipped by TMA on store.
@@ -28,8 +28,8 @@ template <bool PAIR> struct Ring {
   static constexpr int B_ROWS = PAIR ? BN / 2 : BN;       // rows of W one CTA loads per slice
   static constexpr int B_BYTES = B_ROWS * BK * 2;
 };
-constexpr int GEMM_THREADS = 320;      // warp 0 TMA, warp 1 MMA, warps 2-9 epilogue (two per TMEM lane quadrant)
-constexpr int EPI_THREADS = 256;
+constexpr int GEMM_THREADS = 576;      // warp 0 TMA, warp 1 MMA, warps 2-17 epilogue (four per TMEM lane quadrant)
+constexpr int EPI_THREADS = 512;
 constexpr int EPI_BYTES = 128 * 128;    // one staging buffer: 128 rows x 128 bytes (32 fp32 or 64 bf16 columns)
 constexpr int GEMM_SMEM = 4 * (A_BYTES + BN * BK * 2) + 2 * EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/ + BN * 4 /*bias*/;   // both forms: 192 KB of ring
 
@@ -242,9 +242,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     // residual is never read here and every global access is a whole 128-byte row segment.
     constexpr bool F32 = epi_is_f32(EPI);
     constexpr int CW = F32 ? 32 : 64;            // columns per chunk
-    constexpr int TW = CW / 2;                   // columns per thread: two threads share a row
+    constexpr int TW = CW / 4;                   // columns per thread: four threads share a row
     const int q = warp & 3;                      // TMEM lane quadrant this warp may read
-    const int half = (warp - 2) >> 2;            // which half of the chunk's columns
+    const int half = (warp - 2) >> 2;            // which quarter of the chunk's columns
     const int row = q * 32 + lane;
     const bool issuer = threadIdx.x == 64;
     uint32_t tcount = 0, ec = 0;
@@ -259,7 +259,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       // first barrier of the chunk loop publishes the new ones.
       if (ep.bias) {
         const int tcol = threadIdx.x - 64;
-        s_bias[tcol] = n_base + tcol < N ? __ldg(ep.bias + n_base + tcol) : 0.f;
+        if (tcol < BN) s_bias[tcol] = n_base + tcol < N ? __ldg(ep.bias + n_base + tcol) : 0.f;
       }
       mbar_wait(&acc_full[a], (tcount >> 1) & 1, abort_flag, status, 0x400 + a);
       tc_fence_after();
@@ -270,10 +270,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         if (n0 >= N) break;
         uint8_t* buf = sE + (ec & 1) * EPI_BYTES;
         if (issuer) bulk_wait_read<1>();         // the store that last used this buffer has read it
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+        asm volatile("bar.sync 1, 512;" ::: "memory");
         uint32_t acc[TW];
-        if constexpr (F32) tmem_ld16(taddr + c * CW + half * TW, acc);
-        else tmem_ld32(taddr + c * CW + half * TW, acc);
+        if constexpr (F32) tmem_ld8(taddr + c * CW + half * TW, acc);
+        else tmem_ld16(taddr + c * CW + half * TW, acc);
         tc_wait_ld();
 #pragma unroll
         for (int g = 0; g < TW / 8; ++g) {
@@ -286,18 +286,18 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             for (int i = 0; i < 8; ++i) v[i] = 0.f;
           }
           if constexpr (F32) {
-            const int c16 = 4 * half + 2 * g;
+            const int c16 = 2 * half + 2 * g;
             *reinterpret_cast<float4*>(buf + row * 128 + ((c16 ^ (row & 7)) << 4)) = make_float4(v[0], v[1], v[2], v[3]);
             *reinterpret_cast<float4*>(buf + row * 128 + (((c16 + 1) ^ (row & 7)) << 4)) = make_float4(v[4], v[5], v[6], v[7]);
           } else {
             uint4 w;
             w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
             w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
-            *reinterpret_cast<uint4*>(buf + row * 128 + (((4 * half + g) ^ (row & 7)) << 4)) = w;
+            *reinterpret_cast<uint4*>(buf + row * 128 + (((2 * half + g) ^ (row & 7)) << 4)) = w;
           }
         }
         fence_async_smem();
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+        asm volatile("bar.sync 1, 512;" ::: "memory");
         if (issuer && m_base < M) {          // (the odd CTA's half of the last row tile may lie past M)
           if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID) tma_reduce_add_2d(&tm_out, buf, n0, m_base);
           else tma_store_2d(&tm_out, buf, n0, m_base);
