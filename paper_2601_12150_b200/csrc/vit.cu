@@ -71,6 +71,26 @@ __global__ void __launch_bounds__(256) vit_im2col(const float* __restrict__ imag
   a[((int64_t)b * gh * gw + t) * kpad + (c * P + y % P) * P + x % P] = __float2bfloat16(v);
 }
 
+// The same for patch sizes that are multiples of 8: one thread per 8 pixels of a patch row
+// (two 128-bit loads, one 128-bit store).
+__global__ void __launch_bounds__(256) vit_im2col_x8(const float* __restrict__ image, int P, int gh, int gw,
+                                                     const int32_t* __restrict__ bm_of_pos, int kpad,
+                                                     __nv_bfloat16* __restrict__ a) {
+  const int wpix = gw * P, hpix = gh * P;
+  const int x = (blockIdx.x * blockDim.x + threadIdx.x) * 8;
+  const int y = blockIdx.y;
+  const int bc = blockIdx.z;          // b * 3 + c
+  if (x >= wpix) return;
+  const int b = bc / 3, c = bc % 3;
+  const float4* src = reinterpret_cast<const float4*>(image + ((int64_t)bc * hpix + y) * wpix + x);
+  const float4 v0 = __ldcs(src), v1 = __ldcs(src + 1);
+  const int t = __ldg(bm_of_pos + (y / P) * gw + x / P);
+  uint4 o;
+  o.x = spv::pack_bf16(v0.x, v0.y); o.y = spv::pack_bf16(v0.z, v0.w);
+  o.z = spv::pack_bf16(v1.x, v1.y); o.w = spv::pack_bf16(v1.z, v1.w);
+  *reinterpret_cast<uint4*>(a + ((int64_t)b * gh * gw + t) * kpad + (c * P + y % P) * P + x % P) = o;
+}
+
 // Zero the padding columns kp .. kpad-1 of a [rows, kpad] bf16 matrix.
 __global__ void vit_zero_pad(__nv_bfloat16* __restrict__ a, int64_t rows, int kp, int kpad) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -288,8 +308,12 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
   vit_permute_pos<<<cdiv((int64_t)np0 * (D / 4), 256), 256, 0, stream>>>((const float4*)w->pos, bm_pos, G, np0,
                                                                           D / 4, (float4*)pos_bm);
   vit_global_rows<<<dim3(cdiv(G * D, 256), batch), 256, 0, stream>>>(w->cls, w->pos, G, D, L.n0, x);
-  vit_im2col<<<dim3(cdiv(gw * P, 256), gh * P, batch * 3), 256, 0, stream>>>(image, P, gh, gw, bm_of_pos, L.kpad,
-                                                                            acol);
+  if (P % 8 == 0)
+    vit_im2col_x8<<<dim3(cdiv(gw * P / 8, 256), gh * P, batch * 3), 256, 0, stream>>>(image, P, gh, gw, bm_of_pos,
+                                                                                     L.kpad, acol);
+  else
+    vit_im2col<<<dim3(cdiv(gw * P, 256), gh * P, batch * 3), 256, 0, stream>>>(image, P, gh, gw, bm_of_pos, L.kpad,
+                                                                              acol);
   int launches = 4;
   const void* w_pe = w->w_pe;
   if (L.kpad != L.kp) {
