@@ -11,6 +11,7 @@
 //   warp 0      TMA producer (A and W slices, 128-byte swizzle)
 //   warp 1      tcgen05.mma issuer (one thread), owns the TMEM allocation (2 x 256 columns, so
 //               the epilogue of tile i overlaps the main loop of tile i+1)
+//   warp 18     hands staged chunks to TMA (tile store or fp32 add-reduce) and returns the buffers
 //   warps 2..17 epilogue, four threads per output row: TMEM -> registers -> bias / activation /
 //               scale -> swizzled staging buffer -> TMA tile store (bf16 outputs, fp32 rows) or
 //               fp32 TMA add-reduce into the residual stream
@@ -28,8 +29,13 @@ template <bool PAIR> struct Ring {
   static constexpr int B_ROWS = PAIR ? BN / 2 : BN;       // rows of W one CTA loads per slice
   static constexpr int B_BYTES = B_ROWS * BK * 2;
 };
-constexpr int GEMM_THREADS = 576;      // warp 0 TMA, warp 1 MMA, warps 2-17 epilogue (four per TMEM lane quadrant)
+constexpr int GEMM_THREADS = 608;      // warp 0 TMA, warp 1 MMA, warps 2-17 epilogue (four per TMEM lane quadrant),
+                                       // warp 18 hands the staged chunks to TMA
 constexpr int EPI_THREADS = 512;
+constexpr int STORE_WARP = 18;
+// named barriers (0 is __syncthreads): staging buffer b is FULL (written) / EMPTY (read by TMA); the 512
+// epilogue threads and the 32 threads of the store warp take part in each
+constexpr int BAR_FULL = 1, BAR_EMPTY = 3, BAR_EPI = 5, BAR_HANDOFF_THREADS = EPI_THREADS + 32;
 constexpr int EPI_BYTES = 128 * 128;    // one staging buffer: 128 rows x 128 bytes (32 fp32 or 64 bf16 columns)
 constexpr int GEMM_SMEM = 4 * (A_BYTES + BN * BK * 2) + 2 * EPI_BYTES + 1024 /*align*/ + 256 /*barriers*/ + BN * 4 /*bias*/;   // both forms: 192 KB of ring
 
@@ -49,30 +55,31 @@ struct EpiParams {
 // (|error| <= 1.5e-7, branch-free: one reciprocal, one exponential, five multiply-adds), which keeps
 // the epilogue of the MLP GEMM shorter than its main loop; the absolute error of the GELU value is
 // below |x| * 1e-7, far inside the bf16 rounding of the stored activation.
-// Two values at a time: the multiply-adds run as packed fp32x2 instructions.
+// Two values at a time: the multiply-adds run as packed fp32x2 instructions.  Written for the fewest
+// instructions (the epilogue warps of the first MLP GEMM are bound by their issue slots):
+//   gelu(x) = 0.5 x + |x| h,  h = 0.5 erf(|x| / sqrt 2) = 0.5 + q(t) e,
+//   t = 1 / (1 + (p / sqrt 2) |x|),  e = exp(-x^2 / 2) = 2^(-(log2 e / 2) x^2),
+//   q(t) = -0.5 (a1 t + a2 t^2 + a3 t^3 + a4 t^4 + a5 t^5)   (the factor folded into the coefficients).
 __device__ __forceinline__ float2 gelu_erf2(float2 x) {
   const float2 ax = make_float2(fabsf(x.x), fabsf(x.y));
-  const float2 z = __fmul2_rn(ax, make_float2(0.70710678118654752f, 0.70710678118654752f));
-  const float2 den = __ffma2_rn(make_float2(0.3275911f, 0.3275911f), z, make_float2(1.0f, 1.0f));
-  // one reciprocal for the pair: 1/a = b / (a b), 1/b = a / (a b)  (a, b in [1, 1 + 0.23 |x|]); the
-  // special-function unit, at two operations per value, is what bounds this epilogue
+  const float2 den = __ffma2_rn(ax, make_float2(0.3275911f * 0.70710678118654752f, 0.3275911f * 0.70710678118654752f),
+                                make_float2(1.0f, 1.0f));
+  // one reciprocal for the pair: 1/a = b / (a b), 1/b = a / (a b)  (a, b in [1, 1 + 0.23 |x|])
   float r;
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(den.x * den.y));
   const float2 t = __fmul2_rn(make_float2(den.y, den.x), make_float2(r, r));
-  float2 poly = __ffma2_rn(make_float2(1.061405429f, 1.061405429f), t, make_float2(-1.453152027f, -1.453152027f));
-  poly = __ffma2_rn(poly, t, make_float2(1.421413741f, 1.421413741f));
-  poly = __ffma2_rn(poly, t, make_float2(-0.284496736f, -0.284496736f));
-  poly = __ffma2_rn(poly, t, make_float2(0.254829592f, 0.254829592f));
-  poly = __fmul2_rn(poly, t);
-  const float2 arg = __fmul2_rn(__fmul2_rn(z, z), make_float2(-1.4426950408889634f, -1.4426950408889634f));
+  float2 q = __ffma2_rn(make_float2(-0.5f * 1.061405429f, -0.5f * 1.061405429f), t,
+                        make_float2(0.5f * 1.453152027f, 0.5f * 1.453152027f));
+  q = __ffma2_rn(q, t, make_float2(-0.5f * 1.421413741f, -0.5f * 1.421413741f));
+  q = __ffma2_rn(q, t, make_float2(0.5f * 0.284496736f, 0.5f * 0.284496736f));
+  q = __ffma2_rn(q, t, make_float2(-0.5f * 0.254829592f, -0.5f * 0.254829592f));
+  q = __fmul2_rn(q, t);
+  const float2 arg = __fmul2_rn(__fmul2_rn(x, x), make_float2(-0.72134752044448170f, -0.72134752044448170f));
   float2 e;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(arg.x));
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(arg.y));
-  const float2 neg_poly = make_float2(-poly.x, -poly.y);
-  const float2 erf_abs = __ffma2_rn(neg_poly, e, make_float2(1.0f, 1.0f));        // erf(|x| / sqrt 2)
-  const float2 half_x = __fmul2_rn(x, make_float2(0.5f, 0.5f));
-  // 0.5 x (1 + sign(x) erf(|x|/sqrt 2))
-  return __ffma2_rn(make_float2(fabsf(half_x.x), fabsf(half_x.y)), erf_abs, half_x);
+  const float2 h = __ffma2_rn(q, e, make_float2(0.5f, 0.5f));                    // 0.5 erf(|x| / sqrt 2)
+  return __ffma2_rn(ax, h, __fmul2_rn(x, make_float2(0.5f, 0.5f)));             // 0.5 x + |x| h
 }
 // x * sigmoid(x) with the hardware exponential and reciprocal (relative error about 1e-6, far
 // inside the bf16 rounding of the stored value); exp(-x) = inf for x < -88 gives 1/inf = 0, so x * 0 = -0
@@ -133,6 +140,13 @@ __device__ __forceinline__ void epilogue_math(const EpiParams& p, const float* t
     v[0] += a0.x; v[1] += a0.y; v[2] += a0.z; v[3] += a0.w;
     v[4] += a1.x; v[5] += a1.y; v[6] += a1.z; v[7] += a1.w;
   }
+}
+
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void named_bar_arrive(int id, int threads) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 template <int EPI, bool PAIR>
@@ -235,18 +249,44 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         else tc_commit(&acc_full[a]);
       }
     }
+  } else if (warp == STORE_WARP) {
+    // Store warp: waits until the epilogue threads have written a staging buffer, hands it to TMA
+    // (a plain tile store, or an fp32 add into the residual stream, so that the residual is never
+    // read here and every global access is a whole 128-byte row segment), and gives the buffer
+    // back once TMA has read it.  The epilogue threads never wait for one another, only for a buffer.
+    constexpr int CW = epi_is_f32(EPI) ? 32 : 64;
+    uint32_t ec = 0;
+    for (int tile = worker; tile < tiles; tile += n_workers) {
+      const int m_base = (tile / n_tiles) * TILE_M + (int)rank * BM, n_base = (tile % n_tiles) * BN;
+#pragma unroll 1
+      for (int c = 0; c < BN / CW; ++c, ++ec) {
+        const int n0 = n_base + c * CW;
+        if (n0 >= N) break;
+        const int bsel = ec & 1;
+        named_bar_sync(BAR_FULL + bsel, BAR_HANDOFF_THREADS);
+        if (lane == 0) {
+          if (m_base < M) {                  // (the odd CTA's half of the last row tile may lie past M)
+            uint8_t* buf = sE + bsel * EPI_BYTES;
+            if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID) tma_reduce_add_2d(&tm_out, buf, n0, m_base);
+            else tma_store_2d(&tm_out, buf, n0, m_base);
+            bulk_commit();
+            bulk_wait_read<0>();
+          }
+        }
+        __syncwarp();
+        named_bar_arrive(BAR_EMPTY + bsel, BAR_HANDOFF_THREADS);
+      }
+    }
+    if (lane == 0) bulk_wait<0>();
   } else {
     // Epilogue: thread = output row.  A chunk of columns (32 fp32 or 64 bf16 = 128 bytes per row)
-    // goes TMEM -> registers -> arithmetic -> swizzled staging buffer, and one thread hands the
-    // buffer to TMA: a plain tile store, or an fp32 add into the residual stream, so that the
-    // residual is never read here and every global access is a whole 128-byte row segment.
+    // goes TMEM -> registers -> arithmetic -> swizzled staging buffer.
     constexpr bool F32 = epi_is_f32(EPI);
     constexpr int CW = F32 ? 32 : 64;            // columns per chunk
     constexpr int TW = CW / 4;                   // columns per thread: four threads share a row
     const int q = warp & 3;                      // TMEM lane quadrant this warp may read
     const int half = (warp - 2) >> 2;            // which quarter of the chunk's columns
     const int row = q * 32 + lane;
-    const bool issuer = threadIdx.x == 64;
     uint32_t tcount = 0, ec = 0;
     const uint32_t acc_empty_remote = PAIR ? mapa_shared(smem_u32(&acc_empty[0]), 0) : 0u;
     for (int tile = worker; tile < tiles; tile += n_workers, ++tcount) {
@@ -254,12 +294,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       const int m_base = (tile / n_tiles) * TILE_M + (int)rank * BM, n_base = (tile % n_tiles) * BN;
       const int m = m_base + row;
       // the tile's bias goes to shared memory while the main loop still runs: a global load per
-      // chunk would sit (with its L2 latency) on the epilogue's critical path.  Every thread is past
-      // the last barrier of the previous tile here, so nobody still reads the old values; the
-      // first barrier of the chunk loop publishes the new ones.
+      // chunk would sit (with its L2 latency) on the epilogue's critical path.  The barrier before
+      // the fill waits for the slowest thread's last read of the previous tile's values, the one
+      // after it publishes the new ones.
       if (ep.bias) {
+        named_bar_sync(BAR_EPI, EPI_THREADS);
         const int tcol = threadIdx.x - 64;
         if (tcol < BN) s_bias[tcol] = n_base + tcol < N ? __ldg(ep.bias + n_base + tcol) : 0.f;
+        named_bar_sync(BAR_EPI, EPI_THREADS);
       }
       mbar_wait(&acc_full[a], (tcount >> 1) & 1, abort_flag, status, 0x400 + a);
       tc_fence_after();
@@ -269,12 +311,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         const int n0 = n_base + c * CW;
         if (n0 >= N) break;
         uint8_t* buf = sE + (ec & 1) * EPI_BYTES;
-        if (issuer) bulk_wait_read<1>();         // the store that last used this buffer has read it
-        asm volatile("bar.sync 1, 512;" ::: "memory");
         uint32_t acc[TW];
         if constexpr (F32) tmem_ld8(taddr + c * CW + half * TW, acc);
         else tmem_ld16(taddr + c * CW + half * TW, acc);
         tc_wait_ld();
+        uint4 o[TW / (F32 ? 4 : 8)];             // this thread's share of the staged row
 #pragma unroll
         for (int g = 0; g < TW / 8; ++g) {
           float v[8];
@@ -286,29 +327,27 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             for (int i = 0; i < 8; ++i) v[i] = 0.f;
           }
           if constexpr (F32) {
-            const int c16 = 2 * half + 2 * g;
-            *reinterpret_cast<float4*>(buf + row * 128 + ((c16 ^ (row & 7)) << 4)) = make_float4(v[0], v[1], v[2], v[3]);
-            *reinterpret_cast<float4*>(buf + row * 128 + (((c16 + 1) ^ (row & 7)) << 4)) = make_float4(v[4], v[5], v[6], v[7]);
+            o[2 * g] = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+            o[2 * g + 1] = make_uint4(__float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7]));
           } else {
-            uint4 w;
-            w.x = pack_bf16(v[0], v[1]); w.y = pack_bf16(v[2], v[3]);
-            w.z = pack_bf16(v[4], v[5]); w.w = pack_bf16(v[6], v[7]);
-            *reinterpret_cast<uint4*>(buf + row * 128 + (((2 * half + g) ^ (row & 7)) << 4)) = w;
+            o[g] = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
           }
         }
+        // the arithmetic is done before the buffer is needed: TMA has read its previous contents
+        if (ec >= 2) named_bar_sync(BAR_EMPTY + (ec & 1), BAR_HANDOFF_THREADS);
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+          *reinterpret_cast<uint4*>(buf + row * 128 + (((2 * half + j) ^ (row & 7)) << 4)) = o[j];
         fence_async_smem();
-        asm volatile("bar.sync 1, 512;" ::: "memory");
-        if (issuer && m_base < M) {          // (the odd CTA's half of the last row tile may lie past M)
-          if constexpr (EPI == SPV_EPI_BIAS_SCALE_RESID) tma_reduce_add_2d(&tm_out, buf, n0, m_base);
-          else tma_store_2d(&tm_out, buf, n0, m_base);
-          bulk_commit();
-        }
+        named_bar_arrive(BAR_FULL + (ec & 1), BAR_HANDOFF_THREADS);
       }
       tc_fence_before();
       if constexpr (PAIR) mbar_arrive_cluster(acc_empty_remote + 8u * (uint32_t)a);
       else mbar_arrive(&acc_empty[a]);
     }
-    if (issuer) bulk_wait<0>();
+    // take the store warp's last hand-backs, so that no barrier is left half way at exit
+    if (ec >= 2) named_bar_sync(BAR_EMPTY + (ec & 1), BAR_HANDOFF_THREADS);
+    if (ec >= 1) named_bar_sync(BAR_EMPTY + ((ec - 1) & 1), BAR_HANDOFF_THREADS);
   }
   tc_fence_before();
   __syncthreads();
