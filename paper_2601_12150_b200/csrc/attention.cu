@@ -509,15 +509,16 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       }
 #pragma unroll 1
       for (int g = 0; g < G; ++g) {
-        float d[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};     // eight independent chains
+        float2 d[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
+        for (int c = 0; c < 8; ++c) {                              // eight independent chains, packed in pairs
           float kf[8];
           unpack8(*reinterpret_cast<const uint4*>(sKg + g * 128 + ((c ^ (g & 7)) << 4)), kf);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) d[i] = fmaf(qf[8 * c + i], kf[i], d[i]);
+          for (int i = 0; i < 4; ++i)
+            d[i] = __ffma2_rn(make_float2(qf[8 * c + 2 * i], qf[8 * c + 2 * i + 1]), make_float2(kf[2 * i], kf[2 * i + 1]), d[i]);
         }
-        const float sc = (((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]))) * sl2;
+        const float sc = (((d[0].x + d[0].y) + (d[1].x + d[1].y)) + ((d[2].x + d[2].y) + (d[3].x + d[3].y))) * sl2;
         s_sg[g * 128 + row] = sc;
         m_g = fmaxf(m_g, sc);
       }
@@ -557,7 +558,11 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         float vf[8];
         unpack8(*reinterpret_cast<const uint4*>(sVg + g * 128 + ((c ^ (g & 7)) << 4)), vf);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) of[8 * c + i] = fmaf(w, vf[i], of[8 * c + i]);
+        for (int i = 0; i < 8; i += 2) {
+          const float2 t = __ffma2_rn(make_float2(w, w), make_float2(vf[i], vf[i + 1]), make_float2(of[8 * c + i], of[8 * c + i + 1]));
+          of[8 * c + i] = t.x;
+          of[8 * c + i + 1] = t.y;
+        }
       }
     }
     // stage the bf16 row in the (now dead) Q tile, same 128-byte swizzle; each warp then stores its
