@@ -236,7 +236,8 @@ __device__ __forceinline__ void unpack8(const uint4& u, float* f) {
 __global__ void __launch_bounds__(ATT_THREADS, 3)
 attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kg,
-                  const __grid_constant__ CUtensorMap tm_vg, const PatchParams p) {
+                  const __grid_constant__ CUtensorMap tm_vg, const __grid_constant__ CUtensorMap tm_o,
+                  const PatchParams p) {
   const int b = blockIdx.z, h = blockIdx.y;
   const int4 tile = __ldg(p.tiles + (size_t)b * p.tiles_per_image + blockIdx.x);
   const int q_begin = tile.x, q_end = tile.y;
@@ -578,21 +579,33 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         *reinterpret_cast<uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4)) = w;
       }
     }
-    __syncwarp();
-    {
-      const int r0 = 32 * warp + (lane >> 3), cc = lane & 7;
-      __nv_bfloat16* obase = p.o + b * p.o_sb + (int64_t)G * p.o_st + (int64_t)h * p.o_sh + cc * 8;
-      uint4 w[8];
-      int ot[8];
-#pragma unroll
-      for (int q4 = 0; q4 < 8; ++q4) {
-        const int rr = r0 + 4 * q4, tk = q_begin + rr;
-        w[q4] = *reinterpret_cast<const uint4*>(sQ + rr * 128 + ((cc ^ (rr & 7)) << 4));
-        ot[q4] = (p.o_tok && tk < q_end) ? __ldg(p.o_tok + (size_t)b * p.n_patch + tk) : tk;
+    if (p.o_tok == nullptr && 32 * warp + 32 <= q_end - q_begin) {
+      // all 32 rows of this warp are valid and consecutive in the output: one TMA tile store of the
+      // warp's staged rows (four swizzle atoms of eight rows), no waiting for the other warps
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_4d(&tm_o, sQ + warp * (32 * 128), 0, G + q_begin + 32 * warp, h, b);
+        bulk_commit();
+        bulk_wait_read<0>();
       }
+    } else {
+      __syncwarp();
+      {
+        const int r0 = 32 * warp + (lane >> 3), cc = lane & 7;
+        __nv_bfloat16* obase = p.o + b * p.o_sb + (int64_t)G * p.o_st + (int64_t)h * p.o_sh + cc * 8;
+        uint4 w[8];
+        int ot[8];
 #pragma unroll
-      for (int q4 = 0; q4 < 8; ++q4)
-        if (q_begin + r0 + 4 * q4 < q_end) *reinterpret_cast<uint4*>(obase + (int64_t)ot[q4] * p.o_st) = w[q4];
+        for (int q4 = 0; q4 < 8; ++q4) {
+          const int rr = r0 + 4 * q4, tk = q_begin + rr;
+          w[q4] = *reinterpret_cast<const uint4*>(sQ + rr * 128 + ((cc ^ (rr & 7)) << 4));
+          ot[q4] = (p.o_tok && tk < q_end) ? __ldg(p.o_tok + (size_t)b * p.n_patch + tk) : tk;
+        }
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4)
+          if (q_begin + r0 + 4 * q4 < q_end) *reinterpret_cast<uint4*>(obase + (int64_t)ot[q4] * p.o_st) = w[q4];
+      }
     }
   }
   tc_fence_before();
@@ -874,7 +887,10 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   pp.status = ctx->d_status;
   const dim3 grid(plan->tiles_per_image, io->heads, plan->batch);
   SpvProfScope prof(ctx, SPV_K_ATTN_PATCH, stream);
-  attn_patch_kernel<<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, tkg, tvg, pp);
+  // the output as a tensor map (same row order as Q, boxes of 32 rows): warps whose rows are all valid store by TMA
+  CUtensorMap to;
+  if ((st = make_qkv_map(ctx, &to, io->o, io->o_sb, io->o_st, io->o_sh, n_tok, io->heads, plan->batch, 32)) != SPV_OK) return st;
+  attn_patch_kernel<<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, tkg, tvg, to, pp);
   return spv_launch_ok(ctx);
 }
 
