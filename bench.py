@@ -105,7 +105,7 @@ def forward_flops(wl, kept_positions):
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per GEMM launch, averaged over the 104
 # GEMM launches of one step, from one ncu capture (profiles/gemm_dram_vitl16_2048_b4.md).  Valid
 # only for the kernel source it was taken with: reported as null once gemm.cu has changed.
-GEMM_TRAFFIC = {"vitl16_2048_b4_sparse_filter": (376.4e6, "7cd6c9990a76")}
+GEMM_TRAFFIC = {"vitl16_2048_b4_sparse_filter": (375.5e6, "39d36c0b6203")}
 
 
 def gemm_traffic(workload):

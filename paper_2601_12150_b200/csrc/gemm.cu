@@ -320,7 +320,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         for (int g = 0; g < TW / 8; ++g) {
           float v[8];
           const int n = n0 + half * TW + 8 * g;
-          if (m < M && n < N) {
+          // rows past M hold zeros (TMA fills them on load) and are clipped by TMA on store, so only
+          // the epilogue that addresses global memory by row needs the per-lane row guard; without
+          // it the groups are straight-line code and their dependency chains interleave
+          if ((EPI != SPV_EPI_BIAS_MUL || m < M) && n < N) {
             epilogue_math<EPI>(ep, s_bias, n_base, m, n, acc + 8 * g, v);
           } else {
 #pragma unroll
