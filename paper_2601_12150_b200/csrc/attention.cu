@@ -628,7 +628,7 @@ constexpr int GCH = 128;   // fewest keys per CTA (bounds the number of chunk pa
 // followed by a value pass -- and the 32 group states are merged through shared memory.  Writes the
 // chunk's (max, sum, sum p*v) and, when the scores are wanted, the scaled logits.
 template <bool kLogits>
-__global__ void __launch_bounds__(256, 3) attn_global_partial(const __nv_bfloat16* __restrict__ q,
+__global__ void __launch_bounds__(256, 2) attn_global_partial(const __nv_bfloat16* __restrict__ q,
                                                            const __nv_bfloat16* __restrict__ k,
                                                            const __nv_bfloat16* __restrict__ v, int64_t sb,
                                                            int64_t st, int64_t sh, int n_tok, int n_global,
@@ -651,9 +651,8 @@ __global__ void __launch_bounds__(256, 3) attn_global_partial(const __nv_bfloat1
   // end of the chunk are predicated off.  The loads of GU keys (key and value rows) are issued
   // before any of them is used.
   constexpr int GU = 4;
-#pragma unroll 1
-  for (int kk0 = k0; kk0 < k1; kk0 += 32 * GU) {
-    uint4 ku[GU], vu[GU];
+  // the loads of the next GU keys are in flight while the current ones are used
+  auto load_batch = [&](int kk0, uint4* ku, uint4* vu) {
 #pragma unroll
     for (int u = 0; u < GU; ++u) {
       const int kk = kk0 + u * 32 + grp;
@@ -665,6 +664,15 @@ __global__ void __launch_bounds__(256, 3) attn_global_partial(const __nv_bfloat1
         vu[u] = __ldg(reinterpret_cast<const uint4*>(v + off) + sub);
       }
     }
+  };
+  uint4 kn[GU], vn[GU];
+  load_batch(k0, kn, vn);
+#pragma unroll 1
+  for (int kk0 = k0; kk0 < k1; kk0 += 32 * GU) {
+    uint4 ku[GU], vu[GU];
+#pragma unroll
+    for (int u = 0; u < GU; ++u) { ku[u] = kn[u]; vu[u] = vn[u]; }
+    if (kk0 + 32 * GU < k1) load_batch(kk0 + 32 * GU, kn, vn);
     float d[GU];
 #pragma unroll
     for (int u = 0; u < GU; ++u) {
@@ -906,9 +914,9 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   const int n_tok = plan->n_global + plan->n_patch, G = plan->n_global, B = plan->batch;
   if (ws_bytes < spv_attn_global_bytes(B, G, io->heads, n_tok)) return SPV_ERR_WORKSPACE;
   const size_t rows = (size_t)B * G * io->heads;
-  // as many chunks as fill the GPU once (three CTAs of this kernel per SM), none shorter than GCH keys
+  // as many chunks as fill the GPU once (two CTAs of this kernel per SM), none shorter than GCH keys
   const int max_chunks = (n_tok + GCH - 1) / GCH;
-  int chunks = (int)((size_t)ctx->sm_count * 3 / rows);
+  int chunks = (int)((size_t)ctx->sm_count * 2 / rows);
   chunks = chunks < 1 ? 1 : (chunks > max_chunks ? max_chunks : chunks);
   const int chunk_len = ((n_tok + chunks - 1) / chunks + 127) / 128 * 128;
   chunks = (n_tok + chunk_len - 1) / chunk_len;
