@@ -192,3 +192,44 @@ def test_blocks_larger_than_many_tiles(ctx):
         got, _ = _run(ctx, q, k, v, gh, gw, 64, r, scores=False)
         want, _ = oracle.attention(q, k, v, gh, gw, 64, r, rows=rows)
         _check(got[:, rows], want[:, rows])
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_geometries_both_token_orders(ctx, seed):
+    """Seeded random grids, block sizes, radii, global-token counts and kept sets (none, sparse, dense),
+    each run in row-major order and in block-major order (the order used inside vit_forward, where full
+    warps store their rows with TMA and ragged warps row by row), against the oracle."""
+    rng = np.random.default_rng(100 + seed)
+    gh, gw = int(rng.integers(3, 48)), int(rng.integers(3, 48))
+    b = int(rng.choice([1, 2, 3, 4, 7, 8, 16]))
+    r = int(rng.choice([0, 1, 1, 2, 3]))
+    G = int(rng.choice([1, 1, 2, 8]))
+    B, H = int(rng.integers(1, 3)), int(rng.integers(1, 4))
+    keep = rng.choice([0.0, 0.0, 0.3, 0.5, 0.9])
+    n0 = gh * gw
+    if keep == 0.0:
+        pos = np.tile(np.arange(n0, dtype=np.int32), (B, 1))
+        have_pos = False
+    else:
+        kcount = max(1, int(n0 * keep))
+        pos = np.stack([np.sort(rng.choice(n0, size=kcount, replace=False)) for _ in range(B)]).astype(np.int32)
+        have_pos = True
+    n = G + pos.shape[1]
+    q, k, v = synth.attention_qkv(200 + seed, B, n, H, 64)
+    want, wsc = oracle.attention(q, k, v, gh, gw, b, r, n_global=G, patch_pos=pos if have_pos else None,
+                                 want_scores=True)
+    got, gsc = _run(ctx, q, k, v, gh, gw, b, r, G=G, patch_pos=pos if have_pos else None)
+    _check(got, want)
+    assert np.abs(gsc - wsc).max() < 1e-3
+    perm = np.stack([np.lexsort((pos[i], (pos[i] % gw) // b, (pos[i] // gw) // b)) for i in range(B)])
+
+    def reorder(a):
+        out = a.copy()
+        for i in range(B):
+            out[i, G:] = a[i, G + perm[i]]
+        return out
+    pos_bm = np.stack([pos[i][perm[i]] for i in range(B)])
+    got_bm, gsc_bm = _run(ctx, reorder(q), reorder(k), reorder(v), gh, gw, b, r, G=G, patch_pos=pos_bm, order=1)
+    _check(got_bm, reorder(want))
+    for i in range(B):
+        assert np.abs(gsc_bm[i] - wsc[i][:, perm[i]]).max() < 1e-3
