@@ -113,3 +113,30 @@ def test_layernorm(ctx, rows, dim):
     y2 = ctx.layernorm(torch.from_numpy(x).to(dev), torch.from_numpy(g).to(dev), torch.from_numpy(b).to(dev),
                        out_row=perm)
     assert torch.equal(y2[perm.long()], y)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_gemm_random_shapes(ctx, seed):
+    """Seeded random M (single CTAs and CTA pairs), N and K (multiples of 8, ragged against the 256 x 256 x 64
+    tiling) with the fp32 residual epilogue, where every mis-addressed tile, k-slice or bias column shows."""
+    import paper_2601_12150_b200 as spv
+    rng = np.random.default_rng(300 + seed)
+    M = int(rng.choice([rng.integers(1, 257), rng.integers(257, 1500), rng.integers(1500, 6000)]))
+    N = 8 * int(rng.integers(1, 140))
+    K = 8 * int(rng.integers(1, 80))
+    a = synth.round_bf16(rng.standard_normal((M, K), dtype=np.float32))
+    w = synth.round_bf16(rng.standard_normal((N, K), dtype=np.float32) * 0.05)
+    bias = rng.standard_normal(N).astype(np.float32)
+    scale = rng.standard_normal(N).astype(np.float32)
+    resid = rng.standard_normal((M, N)).astype(np.float32)
+    dev = ctx.device
+    out = torch.from_numpy(resid.copy()).to(dev)
+    ctx.gemm_bf16(_bf16(dev, a), _bf16(dev, w), out, spv.EPI_BIAS_SCALE_RESID,
+                  bias=torch.from_numpy(bias).to(dev), scale=torch.from_numpy(scale).to(dev))
+    ctx.check()
+    ref = resid + scale[None] * oracle.linear(a, w, bias)
+    assert np.abs(out.cpu().numpy() - ref).max() < 2e-4, (M, N, K)
+    out2 = torch.zeros((M, N), dtype=torch.bfloat16, device=dev)
+    ctx.gemm_bf16(_bf16(dev, a), _bf16(dev, w), out2, spv.EPI_BIAS_GELU, bias=torch.from_numpy(bias).to(dev))
+    ctx.check()
+    _check(out2.float().cpu().numpy(), np.vectorize(oracle.gelu)(oracle.linear(a, w, bias)).astype(np.float32))
