@@ -151,3 +151,30 @@ def test_vit_forward_argument_errors(ctx):
     assert e.value.status == spv.ERR_WORKSPACE
     with pytest.raises(spv.SpvError):
         ctx.vit_forward(dict(ok, filter_layer=2, keep_ratio=0.5), dw, img, 8, 8)                       # beyond the last block
+
+
+def test_vit_forward_in_a_cuda_graph(ctx):
+    """vit_forward only enqueues work on the given stream (kernels, memset, device copies), so after one
+    warm-up call it can be captured in a CUDA graph; the replay reproduces the direct call bit for bit."""
+    arch = synth.vit_tiny(layers=3, dim=128, heads=2, hidden=256, patch=4)
+    gh, gw, B = 16, 20, 2
+    full = dict(arch, attn_mode=synth.ATTN_SPARSE, block=8, radius=1, filter_layer=1, keep_ratio=0.5)
+    w = synth.vit_weights(11, arch, gh, gw, pos_base=4)
+    dw = ctx.make_vit_weights(w)
+    dev = ctx.device
+    img = torch.from_numpy(synth.tissue_batch(12, B, gh * 4, gw * 4)).to(dev)
+    out, kept = ctx.vit_forward(full, dw, img, gh, gw)
+    ctx.check()
+    ref, ref_kept = out.clone(), kept.clone()      # (the context's cached workspace is reused by the captured call)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(graph, stream=s):
+            out2, kept2 = ctx.vit_forward(full, dw, img, gh, gw, out=out, stream=s)
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    ctx.check()
+    assert torch.equal(out, ref)
+    assert torch.equal(kept2, ref_kept)
