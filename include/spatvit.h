@@ -291,6 +291,47 @@ int32_t spv_profile_enable(spv_ctx* ctx, int32_t enable);
  * clear the record. */
 int32_t spv_profile_read(spv_ctx* ctx, spv_kernel_stat* out);
 
+/* ------------------------------------------------------------------------------------------
+ * Hardware rate probes (no counterpart in the paper): the rates the attention kernel's design is
+ * argued from, measured on the device the context was created on.  Each probe runs its kernel twice
+ * and times the second run; the call is synchronous on `stream`.
+ *   SPV_MB_EX2           ex2.approx.ftz.f32, eight independent chains per thread; units = operations
+ *   SPV_MB_SOFTMAX_BODY  inner body of the online softmax on 64 scores per thread (scale, 2^x, row
+ *                        sum, bf16 pack); poly_per_8 in {0, 2, 4, 8} of every eight exponentials are
+ *                        evaluated as a cubic on the multiply-add pipe; units = scores
+ *   SPV_MB_MMA_SS / _TS  tcgen05.mma kind::f16 of m x n x 16 (m 64 or 128, n multiple of 16 up to
+ *                        256), A from shared memory / from TMEM, one issuing thread per CTA, iters x 4
+ *                        instructions rotating over `accumulators` TMEM accumulators; units = FLOP
+ *   SPV_MB_L2_TMA        TMA tile loads of box_rows x 128 bytes from a buffer of at most 32 MB (so
+ *                        that it stays in L2), `stages` loads in flight per CTA; units = bytes
+ * buffer: device scratch, 256-byte aligned; SPV_MB_L2_TMA walks over it (give it 32 MB + 64 KB), the
+ * other probes need 64 KB.  Contents are not preserved.
+ * ---------------------------------------------------------------------------------------- */
+enum { SPV_MB_EX2 = 0, SPV_MB_SOFTMAX_BODY = 1, SPV_MB_MMA_SS = 2, SPV_MB_MMA_TS = 3, SPV_MB_L2_TMA = 4 };
+typedef struct {
+  int32_t kind;
+  int32_t ctas_per_sm; /* grid = SM count x this (1..4)                                          */
+  int32_t threads;     /* per CTA, EX2 / SOFTMAX_BODY only                                       */
+  int32_t iters;       /* loop trips per thread / issuing thread                                 */
+  int32_t m, n;        /* MMA shape                                                              */
+  int32_t box_rows, stages; /* L2_TMA                                                            */
+  int32_t poly_per_8;  /* SOFTMAX_BODY                                                           */
+  int32_t accumulators; /* MMA: consecutive instructions rotate over this many accumulators (1..8;
+                           1 = the dependent chain of a K loop)                                  */
+  int32_t issue_mode;   /* MMA: 0 = one thread alone runs the issue loop; 1 = its whole warp runs the
+                           loop and an elected lane issues                                       */
+  int32_t issuers;      /* MMA: warps of the CTA that issue concurrently, each on its own
+                           accumulators (1..4)                                                   */
+} spv_microbench_desc;
+typedef struct {
+  double ms;      /* CUDA-event time of the timed run                                            */
+  double cycles;  /* SM cycles of the slowest CTA (clock64)                                      */
+  double units;   /* work of the timed run, see above                                            */
+  int32_t sm_count;
+} spv_microbench_result;
+int32_t spv_microbench(spv_ctx* ctx, const spv_microbench_desc* desc, void* buffer, size_t buffer_bytes,
+                       void* stream, spv_microbench_result* out);
+
 #ifdef __cplusplus
 }
 #endif

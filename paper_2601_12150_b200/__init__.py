@@ -23,7 +23,7 @@ EXPORTS = ["spv_create", "spv_destroy", "spv_status_string", "spv_check", "spv_l
            "spv_filter_keep_count", "spv_filter_workspace_size", "cls_score_topk_filter",
            "cls_score_topk_filter_static",
            "spv_vit_workspace_size", "vit_forward", "spv_gemm_bf16", "spv_layernorm",
-           "spv_profile_enable", "spv_profile_read"]
+           "spv_profile_enable", "spv_profile_read", "spv_microbench"]
 
 
 class SpvError(RuntimeError):
@@ -84,6 +84,20 @@ class GemmDesc(C.Structure):
                 ("ldadd", C.c_int64), ("rows_per_image", C.c_int32)]
 
 
+MICROBENCH_KINDS = {"ex2": 0, "softmax_body": 1, "mma_ss": 2, "mma_ts": 3, "l2_tma": 4}
+
+
+class MicrobenchDesc(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("ctas_per_sm", C.c_int32), ("threads", C.c_int32), ("iters", C.c_int32),
+                ("m", C.c_int32), ("n", C.c_int32), ("box_rows", C.c_int32), ("stages", C.c_int32),
+                ("poly_per_8", C.c_int32), ("accumulators", C.c_int32),
+                ("issue_mode", C.c_int32), ("issuers", C.c_int32)]
+
+
+class MicrobenchResult(C.Structure):
+    _fields_ = [("ms", C.c_double), ("cycles", C.c_double), ("units", C.c_double), ("sm_count", C.c_int32)]
+
+
 _lib = None
 
 
@@ -123,6 +137,8 @@ def lib():
                                     C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
         L.spv_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         L.spv_profile_read.argtypes = [C.c_void_p, C.POINTER(KernelStat)]
+        L.spv_microbench.argtypes = [C.c_void_p, C.POINTER(MicrobenchDesc), C.c_void_p, C.c_size_t, C.c_void_p,
+                                     C.POINTER(MicrobenchResult)]
         _lib = L
     return _lib
 
@@ -222,6 +238,18 @@ class Context:
         _raise(lib().spv_profile_read(self.handle, arr), "spv_profile_read")
         return {n: dict(launches=int(a.launches), ms=float(a.ms), work=float(a.work))
                 for n, a in zip(KERNEL_CLASSES, arr)}
+
+    def microbench(self, kind, ctas_per_sm=1, threads=128, iters=1000, m=128, n=64, box_rows=64, stages=4,
+                   poly_per_8=0, accumulators=1, issue_mode=0, issuers=1, stream=None):
+        """One hardware rate probe (spv_microbench); returns dict(ms, cycles, units, sm_count)."""
+        d = MicrobenchDesc(MICROBENCH_KINDS[kind], ctas_per_sm, threads, iters, m, n, box_rows, stages, poly_per_8,
+                           accumulators, issue_mode, issuers)
+        nbytes = (32 << 20) + (64 << 10) if kind == "l2_tma" else (64 << 10)
+        buf = self.workspace(nbytes)
+        r = MicrobenchResult()
+        _raise(lib().spv_microbench(self.handle, C.byref(d), _ptr(buf), buf.numel(), _stream(stream), C.byref(r)),
+               "spv_microbench")
+        return dict(ms=r.ms, cycles=r.cycles, units=r.units, sm_count=r.sm_count)
 
     # -- Sec. 3.3 ---------------------------------------------------------------------------
     def cls_score_topk_filter(self, scores, tokens_in=None, n_global=1, keep_ratio=0.5,
