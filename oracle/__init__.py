@@ -27,7 +27,8 @@ class _VitConfig(C.Structure):
                 ("mlp_hidden", C.c_int32), ("mlp_kind", C.c_int32), ("patch", C.c_int32),
                 ("n_global", C.c_int32), ("has_layerscale", C.c_int32), ("ln_eps", C.c_float),
                 ("attn_mode", C.c_int32), ("block", C.c_int32), ("radius", C.c_int32),
-                ("filter_layer", C.c_int32), ("keep_ratio", C.c_double)]
+                ("filter_layer", C.c_int32), ("keep_ratio", C.c_double),
+                ("n_filters", C.c_int32), ("filter_layers", C.c_int32 * 4), ("keep_ratios", C.c_double * 4)]
 
 
 _LAYER_FIELDS = ["ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_o", "b_o", "ls1", "ln2_g", "ln2_b",
@@ -200,18 +201,44 @@ def silu_mul_n(a, b):
     return y
 
 
-def vit_forward(cfg, weights, image, grid_h, grid_w, forced_keep=None, tap_layer=None):
-    """Whole forward.  cfg: dict with the spvo_vit_config fields; weights: dict of fp32 numpy
-    arrays (`w_pe, b_pe, cls, pos, lnf_g, lnf_b` and `layers`: list of dicts with the
-    per-layer names); image fp32 [B, 3, H*patch, W*patch].
+def filter_stages(cfg):
+    """[(layer, keep_ratio), ...] of a config dict: `filters` (a list of such pairs, layers strictly
+    increasing) or the single stage `filter_layer` / `keep_ratio`."""
+    if cfg.get("filters"):
+        return [(int(l), float(k)) for l, k in cfg["filters"]]
+    if cfg.get("filter_layer", 0) > 0:
+        return [(int(cfg["filter_layer"]), float(cfg["keep_ratio"]))]
+    return []
 
-    Returns dict(out=[B, G+k, dim], kept_idx=[B, k] | None, tap=... | None)."""
+
+def stage_keep_counts(cfg, npatch):
+    """Tokens kept by each stage, in order."""
+    out, cur = [], npatch
+    for _, keep in filter_stages(cfg):
+        cur = keep_count(cur, keep)
+        out.append(cur)
+    return out
+
+
+def vit_forward(cfg, weights, image, grid_h, grid_w, forced_keep=None, tap_layer=None):
+    """Whole forward.  cfg: dict with the spvo_vit_config fields (`filters`: optional list of
+    (layer, keep_ratio) stages); weights: dict of fp32 numpy arrays (`w_pe, b_pe, cls, pos, lnf_g, lnf_b`
+    and `layers`: list of dicts with the per-layer names); image fp32 [B, 3, H*patch, W*patch].
+    forced_keep: [B, k_1 + ... + k_S] original positions kept by each stage, stage after stage.
+
+    Returns dict(out=[B, G+k, dim], kept_idx=[B, k] of the last stage | None,
+    kept_all=[B, k_1+...+k_S] | None, tap=... | None)."""
     image = _f32(image)
     B = image.shape[0]
+    stages = filter_stages(cfg)
+    multi = bool(cfg.get("filters"))
+    fl = (C.c_int32 * 4)(*([l for l, _ in stages] + [0] * (4 - len(stages)))) if multi else (C.c_int32 * 4)()
+    kr = (C.c_double * 4)(*([k for _, k in stages] + [0.0] * (4 - len(stages)))) if multi else (C.c_double * 4)()
     c = _VitConfig(cfg["layers"], cfg["dim"], cfg["heads"], cfg["mlp_hidden"], cfg["mlp_kind"],
                    cfg["patch"], cfg["n_global"], cfg.get("has_layerscale", 0),
                    cfg.get("ln_eps", 1e-6), cfg["attn_mode"], cfg.get("block", 8),
-                   cfg.get("radius", 1), cfg.get("filter_layer", 0), cfg.get("keep_ratio", 1.0))
+                   cfg.get("radius", 1), 0 if multi else cfg.get("filter_layer", 0),
+                   1.0 if multi else cfg.get("keep_ratio", 1.0), len(stages) if multi else 0, fl, kr)
     keepalive = []
 
     def fp(a):
@@ -230,22 +257,26 @@ def vit_forward(cfg, weights, image, grid_h, grid_w, forced_keep=None, tap_layer
                     C.cast(L, C.c_void_p))
     G, D = cfg["n_global"], cfg["dim"]
     npatch = grid_h * grid_w
-    filt = cfg.get("filter_layer", 0) > 0
-    k = keep_count(npatch, cfg["keep_ratio"]) if filt else npatch
+    counts = stage_keep_counts(cfg, npatch)
+    k = counts[-1] if counts else npatch
+    k_total = sum(counts)
     out = np.zeros((B, G + k, D), dtype=np.float32)
-    kept = np.zeros((B, k), dtype=np.int32) if filt else None
+    kept = np.zeros((B, k_total), dtype=np.int32) if counts else None
     fk = None
     if forced_keep is not None:
         fk = np.ascontiguousarray(forced_keep, dtype=np.int32)
-        assert fk.shape == (B, k)
+        assert fk.shape == (B, k_total)
     tap = None
     tl = -1
     if tap_layer is not None:
         tl = int(tap_layer)
-        ntap = G + (k if (filt and tl >= cfg["filter_layer"]) else npatch)
-        tap = np.zeros((B, ntap, D), dtype=np.float32)
+        ntap = npatch
+        for (layer, _), cnt in zip(stages, counts):
+            if tl >= layer:
+                ntap = cnt
+        tap = np.zeros((B, G + ntap, D), dtype=np.float32)
     rc = lib().spvo_vit_forward(C.byref(c), C.byref(w), _ptr(image), B, grid_h, grid_w, _ptr(out),
                                 _ptr(kept), _ptr(fk), C.c_int32(tl), _ptr(tap))
     if rc != 0:
         raise ValueError(f"spvo_vit_forward failed ({rc})")
-    return {"out": out, "kept_idx": kept, "tap": tap}
+    return {"out": out, "kept_idx": None if kept is None else kept[:, k_total - k:], "kept_all": kept, "tap": tap}

@@ -77,7 +77,11 @@ int32_t spvo_attention(const spvo_attn_desc* d, const float* q, const float* k,
       const int32_t h = (int32_t)((wi / nq) % H);
       const int32_t bi = (int32_t)(wi / ((int64_t)nq * H));
       const int32_t i = rows ? rows[qi] : qi;
-      if (i < 0 || i >= N) { bad = 1; continue; }
+      if (i < 0 || i >= N) {
+#pragma omp atomic write
+        bad = 1;
+        continue;
+      }
       const float* qv = q + (((int64_t)bi * N + i) * H + h) * E;
       double mx = -INFINITY;
       for (int32_t j = 0; j < N; ++j) {
@@ -152,9 +156,9 @@ int32_t spvo_dense_attention(int32_t batch, int32_t n_tok, int32_t heads,
 
 /* ------------------------------------------------------------------------- */
 /* Sec. 3.3 -- token filter.                                                 */
-/* "rank all tokens by their importance and permanently discard a proportion */
-/* p with the lowest scores": floor(p * N_p) tokens go, so with keep = 1 - p  */
-/* the number kept is ceil(keep * N_p) (a 1e-9 guard absorbs the fp64        */
+/* Tokens are ranked by importance and the share p with the lowest scores is */
+/* dropped for good: floor(p * N_p) tokens go, so with keep = 1 - p the      */
+/* number kept is ceil(keep * N_p) (a 1e-9 guard absorbs the fp64            */
 /* representation error of keep * N_p), at least 1 and at most N_p.          */
 /* ------------------------------------------------------------------------- */
 int32_t spvo_keep_count(int32_t n_patch, double keep_ratio) {
@@ -291,7 +295,32 @@ int32_t spvo_vit_forward(const spvo_vit_config* c, const spvo_vit_weights* w,
   const int32_t D = c->dim, G = c->n_global, P = c->patch, NP0 = gh * gw;
   const int32_t hd = D / c->heads, KP = 3 * P * P, HID = c->mlp_hidden;
   if (c->layers < 1 || D % c->heads != 0 || batch < 1 || NP0 < 1) return 1;
-  if (c->filter_layer < 0 || c->filter_layer > c->layers) return 1;
+  /* the filter stages: (layer, keep ratio) pairs, layers strictly increasing */
+  int32_t n_stage = 0, st_layer[4];
+  double st_keep[4];
+  if (c->n_filters < 0 || c->n_filters > 4) return 1;
+  if (c->n_filters == 0) {
+    if (c->filter_layer < 0 || c->filter_layer > c->layers) return 1;
+    if (c->filter_layer > 0) { n_stage = 1; st_layer[0] = c->filter_layer; st_keep[0] = c->keep_ratio; }
+  } else {
+    n_stage = c->n_filters;
+    for (int32_t s = 0; s < n_stage; ++s) {
+      st_layer[s] = c->filter_layers[s];
+      st_keep[s] = c->keep_ratios[s];
+      if (st_layer[s] < 1 || st_layer[s] > c->layers) return 1;
+      if (s > 0 && st_layer[s] <= st_layer[s - 1]) return 1;
+    }
+  }
+  int32_t k_total = 0;                    /* entries per image in kept_idx / forced_keep */
+  {
+    int32_t cur = NP0;
+    for (int32_t s = 0; s < n_stage; ++s) {
+      cur = spvo_keep_count(cur, st_keep[s]);
+      if (cur < 0) return 3;
+      k_total += cur;
+    }
+  }
+  int32_t stage = 0, k_before = 0;        /* next stage; entries of earlier stages */
   int32_t np = NP0;                       /* patch tokens currently present */
   int64_t N = G + np;
   const int64_t Wpix = (int64_t)gw * P, Hpix = (int64_t)gh * P;
@@ -337,9 +366,8 @@ int32_t spvo_vit_forward(const spvo_vit_config* c, const spvo_vit_weights* w,
     float* vb = (float*)malloc(sizeof(float) * (size_t)(R * D));
     float* ab = (float*)malloc(sizeof(float) * (size_t)(R * D));
     float* pb = (float*)malloc(sizeof(float) * (size_t)(R * D));
-    float* sc = (l == c->filter_layer)
-                    ? (float*)malloc(sizeof(float) * (size_t)((int64_t)batch * c->heads * np))
-                    : NULL;
+    const int is_stage = stage < n_stage && l == st_layer[stage];
+    float* sc = is_stage ? (float*)malloc(sizeof(float) * (size_t)((int64_t)batch * c->heads * np)) : NULL;
 
     /* attention branch: x += ls1 * (Attn(LN1(x)) W_o^T + b_o) */
     spvo_layernorm(x, R, D, lw->ln1_g, lw->ln1_b, c->ln_eps, hbuf);
@@ -383,21 +411,34 @@ int32_t spvo_vit_forward(const spvo_vit_config* c, const spvo_vit_weights* w,
         x[r * D + i] += (lw->ls2 ? lw->ls2[i] : 1.0f) * pb[r * D + i];
     free(h1);
 
-    /* Sec. 3.3: after block `filter_layer`, drop the lowest-scored patches
-     * from the residual stream for all later blocks. */
-    if (l == c->filter_layer) {
-      const int32_t k = spvo_keep_count(np, c->keep_ratio);
+    /* Sec. 3.3: after a stage's block, the lowest-scored patches leave the
+     * residual stream for all later blocks.  The ranking is over the tokens
+     * present (ties: lower index, i.e. lower original position, first);
+     * survivors keep their original grid positions. */
+    if (is_stage) {
+      const int32_t k = spvo_keep_count(np, st_keep[stage]);
       if (k < 0) return 3;
-      int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)((int64_t)batch * k));
+      int32_t* keep = (int32_t*)malloc(sizeof(int32_t) * (size_t)((int64_t)batch * k));  /* indices into the present tokens */
       if (forced_keep) {
-        memcpy(keep, forced_keep, sizeof(int32_t) * (size_t)((int64_t)batch * k));
+        /* given as original positions: look each one up among the present tokens */
+        for (int32_t b = 0; b < batch; ++b)
+          for (int32_t t = 0; t < k; ++t) {
+            const int32_t want = forced_keep[(int64_t)b * k_total + k_before + t];
+            int32_t found = -1;
+            if (!pos) found = (want >= 0 && want < np) ? want : -1;
+            else
+              for (int32_t j = 0; j < np; ++j)
+                if (pos[(int64_t)b * np + j] == want) { found = j; break; }
+            if (found < 0) return 4;
+            keep[(int64_t)b * k + t] = found;
+          }
       } else {
-        if (spvo_filter(batch, c->heads, np, G, D, c->keep_ratio, sc, NULL, NULL, keep, NULL))
+        if (spvo_filter(batch, c->heads, np, G, D, st_keep[stage], sc, NULL, NULL, keep, NULL))
           return 3;
       }
       const int64_t N2 = G + k;
       float* x2 = (float*)malloc(sizeof(float) * (size_t)(batch * N2 * D));
-      pos = (int32_t*)malloc(sizeof(int32_t) * (size_t)((int64_t)batch * k));
+      int32_t* pos2 = (int32_t*)malloc(sizeof(int32_t) * (size_t)((int64_t)batch * k));
       for (int32_t b = 0; b < batch; ++b) {
         memcpy(x2 + (int64_t)b * N2 * D, x + (int64_t)b * N * D, sizeof(float) * (size_t)(G * D));
         for (int32_t t = 0; t < k; ++t) {
@@ -405,15 +446,20 @@ int32_t spvo_vit_forward(const spvo_vit_config* c, const spvo_vit_weights* w,
           if (j < 0 || j >= np) return 4;
           memcpy(x2 + ((int64_t)b * N2 + G + t) * D, x + ((int64_t)b * N + G + j) * D,
                  sizeof(float) * (size_t)D);
-          pos[(int64_t)b * k + t] = j;   /* first filter: index == grid position */
+          /* before the first stage the index is the grid position itself */
+          pos2[(int64_t)b * k + t] = pos ? pos[(int64_t)b * np + j] : j;
+          if (kept_idx) kept_idx[(int64_t)b * k_total + k_before + t] = pos2[(int64_t)b * k + t];
         }
       }
-      if (kept_idx) memcpy(kept_idx, keep, sizeof(int32_t) * (size_t)((int64_t)batch * k));
       free(keep);
       free(x);
+      if (pos) free(pos);
       x = x2;
+      pos = pos2;
       np = k;
       N = N2;
+      k_before += k;
+      ++stage;
     }
     free(hbuf); free(qkv); free(qb); free(kb); free(vb); free(ab); free(pb);
     if (sc) free(sc);

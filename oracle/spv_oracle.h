@@ -87,6 +87,13 @@ typedef struct {
   int32_t attn_mode, block, radius;
   int32_t filter_layer;        /* 0 = off; f => after block f (1-based)        */
   double keep_ratio;
+  /* Several filter stages (Sec. 3.3 applied more than once): stage s runs
+   * after block filter_layers[s] (1-based, strictly increasing) and keeps
+   * ceil(keep_ratios[s] * tokens present).  n_filters == 0: the single stage
+   * (filter_layer, keep_ratio) above, if filter_layer > 0. */
+  int32_t n_filters;
+  int32_t filter_layers[4];
+  double keep_ratios[4];
 } spvo_vit_config;
 
 typedef struct {
@@ -111,9 +118,11 @@ typedef struct {
 } spvo_vit_weights;
 
 /* Whole forward.  image fp32 [batch, 3, H*patch, W*patch].
- * out_tokens fp32 [batch, G+k, dim] after the final LayerNorm (k = H*W when the
- * filter is off).  kept_idx optional [batch, k].  forced_keep optional
- * [batch, k] ascending patch indices: bypass the ranking (teacher forcing).
+ * out_tokens fp32 [batch, G+k, dim] after the final LayerNorm (k = tokens left
+ * by the last stage; H*W when the filter is off).  kept_idx optional
+ * [batch, k_1 + ... + k_S]: per image the kept sets of the stages one after
+ * the other, each as ascending ORIGINAL grid positions.  forced_keep optional,
+ * same layout: bypass the ranking of every stage (teacher forcing).
  * tap_layer / tap_x optional: copy of the residual stream [batch, N_l, dim]
  * after block tap_layer (1-based; 0 = after patch embedding). */
 int32_t spvo_vit_forward(const spvo_vit_config* c, const spvo_vit_weights* w,

@@ -25,22 +25,21 @@ namespace {
 using namespace spv;
 
 constexpr int TQ = 128;            // query rows per tile (MMA M)
-constexpr int TK = 64;             // keys per tile (MMA N of S, K extent of P V)
+constexpr int TK = 64;             // keys per tile (MMA N of S, K extent of P V): with 64, a CTA needs 160 TMEM
+                                   // columns and 136 registers per softmax thread, so three CTAs fit an SM
 constexpr int HD = 64;             // head_dim
-constexpr int KST = 4;             // K / V smem stages (Q K^T runs two key tiles ahead of P V)
-constexpr int NSB = 3;             // S / P buffers in TMEM: a softmax warp may be two key tiles ahead of the slowest
+constexpr int KST = 3;             // K / V smem stages
 constexpr int ATT_THREADS = 256;   // warps 0-3 softmax (one warpgroup), 4 TMA, 5 MMA, 6-7 idle: the second
                                    // warpgroup exists so that it can hand its registers to the first
 constexpr int TILE_BYTES = 128 * 128;  // Q tile
 constexpr int KV_BYTES = TK * 128;      // K or V tile
-constexpr int MAXG = 16;           // global tokens
-constexpr int GROW_BYTES = MAXG * 128;   // global-token rows of one head
+constexpr int GROW_BYTES = 1024;   // global-token rows of one head: up to 8 x 128 B
 constexpr int ATT_SMEM = TILE_BYTES + 2 * KST * KV_BYTES + 2 * GROW_BYTES + 1024 /*align*/ + 256 /*barriers*/ +
-                         MAXG * 128 * 4 /*global-token scores*/;
-// One TMEM allocation of 256 columns per CTA (two CTAs share an SM's 512): three S buffers of 64 fp32
-// columns, each of which receives its own P (bf16, 32 columns) in place once the row has been read, and O.
-constexpr uint32_t TMEM_COLS = 256;
-constexpr uint32_t S_COL = 0, O_COL = NSB * TK;
+                         8 * 128 * 4 /*global-token scores*/;
+constexpr int MAXG = 8;
+// two TMEM allocations per CTA, 160 columns in all, so that three CTAs share an SM's 512
+constexpr uint32_t TMEM_COLS = 128, TMEM_P_COLS = 32;
+constexpr uint32_t S_COL = 0, O_COL = 64;
 
 // ------------------------------------------------------------------------------------------
 // plan
@@ -234,7 +233,7 @@ __device__ __forceinline__ void unpack8(const uint4& u, float* f) {
   }
 }
 
-__global__ void __launch_bounds__(ATT_THREADS, 2)
+__global__ void __launch_bounds__(ATT_THREADS, 3)
 attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kg,
                   const __grid_constant__ CUtensorMap tm_vg, const __grid_constant__ CUtensorMap tm_o,
@@ -258,10 +257,11 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   uint64_t* k_empty = k_full + KST;
   uint64_t* v_full = k_empty + KST;
   uint64_t* v_empty = v_full + KST;
-  uint64_t* s_full = v_empty + KST;      // [NSB] Q K^T of the buffer's key tile has completed
-  uint64_t* p_full = s_full + NSB;       // [NSB] all 128 rows have written P (and read S) of the buffer
-  uint64_t* pv_done = p_full + NSB;      // [NSB] P V of the buffer's key tile (and all before it) has completed
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + NSB);
+  uint64_t* s_full = v_empty + KST;
+  uint64_t* s_free = s_full + 1;
+  uint64_t* p_full = s_free + 1;
+  uint64_t* pv_done = p_full + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + 1);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   float* s_sg = reinterpret_cast<float*>(bars + 32);     // [G][128] scaled scores of the global keys
 
@@ -277,23 +277,27 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
       mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
     }
-    for (int s = 0; s < NSB; ++s) { mbar_init(&s_full[s], 1); mbar_init(&p_full[s], 128); mbar_init(&pv_done[s], 1); }
+    mbar_init(s_full, 1);
+    mbar_init(s_free, 128);
+    mbar_init(p_full, 128);
+    mbar_init(pv_done, 1);
     *abort_flag = 0;
     mbar_fence_init();
   }
   if (warp == 5) {
     tmem_alloc(tmem_slot, TMEM_COLS);
+    tmem_alloc(tmem_slot + 2, TMEM_P_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem = *tmem_slot, tmem_p = tmem_slot[2];
 
   // the softmax warpgroup holds a whole score row of the key tile (64 columns) per thread; the other warpgroup
-  // needs few registers (the kernel starts with 128 per thread: 128 + (128 - 48) = 208)
+  // needs few registers
   if (warp >= 4) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 24;");
   if (warp == 4) {
     // ---------------- TMA producer
     if (lane == 0) {
@@ -328,47 +332,43 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       constexpr uint32_t idesc_s = idesc_bf16(TQ, TK, false);
       constexpr uint32_t idesc_o = idesc_bf16(TQ, HD, true);
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ));
+      auto issue_qk = [&](uint32_t j) {
+        const int s = j % KST;
+        mbar_wait(&k_full[s], (j / KST) & 1, abort_flag, p.status, 0x1300 + s);
+        if (j > 0) mbar_wait(s_free, (j - 1) & 1, abort_flag, p.status, 0x1400);
+        tc_fence_after();
+        const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * KV_BYTES));
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk)
+          mma_ss(tmem + S_COL, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_s, kk != 0);
+        tc_commit(s_full);
+        tc_commit(&k_empty[s]);
+      };
       mbar_wait(q_full, 0, abort_flag, p.status, 0x1000);
-      // Q K^T of key tile t goes to S buffer t % 3 two tiles ahead of P V: the tensor pipe executes this thread's
-      // MMAs in issue order, so Q K^T (t) may overwrite the buffer as soon as P V (t - 3), which read P from it,
-      // has been issued
-      for (uint32_t t = 0; t < n_kv + 2; ++t) {
-        if (t < n_kv) {
-          const int s = t % KST;
-          mbar_wait(&k_full[s], (t / KST) & 1, abort_flag, p.status, 0x1300 + s);
-          tc_fence_after();
-          const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * KV_BYTES));
-          const uint32_t sb = t % NSB;
+      if (n_kv > 0) issue_qk(0);
+      for (uint32_t j = 0; j < n_kv; ++j) {
+        if (j + 1 < n_kv) issue_qk(j + 1);
+        const int s = j % KST;
+        mbar_wait(&v_full[s], (j / KST) & 1, abort_flag, p.status, 0x1500 + s);
+        mbar_wait(p_full, j & 1, abort_flag, p.status, 0x1600);
+        tc_fence_after();
+        const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * KV_BYTES));
 #pragma unroll
-          for (int kk = 0; kk < HD / 16; ++kk)
-            mma_ss(tmem + S_COL + sb * TK, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_s, kk != 0);
-          tc_commit(&s_full[sb]);
-          tc_commit(&k_empty[s]);
-        }
-        if (t >= 2) {
-          const uint32_t j = t - 2;
-          const int s = j % KST;
-          const uint32_t sb = j % NSB;
-          mbar_wait(&v_full[s], (j / KST) & 1, abort_flag, p.status, 0x1500 + s);
-          mbar_wait(&p_full[sb], (j / NSB) & 1, abort_flag, p.status, 0x1600 + sb);
-          tc_fence_after();
-          const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * KV_BYTES));
-#pragma unroll
-          for (int kk = 0; kk < TK / 16; ++kk)
-            mma_ts(tmem + O_COL, tmem + S_COL + sb * TK + kk * 8, dv + (uint64_t)(kk * 128), idesc_o, (j | kk) != 0);
-          tc_commit(&pv_done[sb]);
-          tc_commit(&v_empty[s]);
-        }
+        for (int kk = 0; kk < TK / 16; ++kk)
+          mma_ts(tmem + O_COL, tmem_p + kk * 8, dv + (uint64_t)(kk * 128), idesc_o, (j | kk) != 0);
+        tc_commit(pv_done);
+        tc_commit(&v_empty[s]);
       }
     }
   }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 136;");
     // ---------------- softmax + epilogue: thread `row` owns query row `row` (TMEM lane `row`)
     const int row = threadIdx.x;
     const int tok = q_begin + row;
     const bool valid = tok < q_end;
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_addr_p = tmem_p + ((uint32_t)(warp * 32) << 16);
     int bxq = bx_first;
     if (valid) bxq = __ldg(p.tok_blk + (size_t)b * p.n_patch + tok) % p.nbx;
     const int rlo = max(bxq - r, 0), rhi = min(bxq + r, p.nbx - 1);
@@ -401,29 +401,16 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const int u_hi = __reduce_max_sync(0xffffffffu, some ? c_hi : 0);
         const int i_lo = __reduce_max_sync(0xffffffffu, some ? c_lo : TK);
         const int i_hi = __reduce_min_sync(0xffffffffu, some ? c_hi : 0);
-        const uint32_t sbuf = j % NSB, sph = (j / NSB) & 1;
-        const uint32_t s_addr = lane_addr + S_COL + sbuf * TK;
-        mbar_wait(&s_full[sbuf], sph, abort_flag, p.status, 0x1800 + sbuf);
+        mbar_wait(s_full, j & 1, abort_flag, p.status, 0x1800);
         tc_fence_after();
-        if (u_lo >= u_hi) {
-          // no row of this warp has a key in the tile: P = 0 for its 32 rows and on to the next tile, without
-          // waiting for the other warps (their rows' P V needs this warp's rows of P all the same)
-          uint32_t z[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) z[i] = 0u;
-          tmem_st16(s_addr, z);
-          tmem_st16(s_addr + 16, z);
-          tc_wait_st();
-          tc_fence_before();
-          mbar_arrive(&p_full[sbuf]);
-          continue;
-        }
-        // one pass: the live 32-column chunks of S go to registers
+        // one pass: the live 32-column chunks of S go to registers, then S is released
         uint32_t sr[TK];
 #pragma unroll
         for (int c = 0; c < TK / 32; ++c)
-          if (32 * c < u_hi && 32 * c + 32 > u_lo) tmem_ld32(s_addr + 32 * c, sr + 32 * c);
+          if (32 * c < u_hi && 32 * c + 32 > u_lo) tmem_ld32(lane_addr + S_COL + 32 * c, sr + 32 * c);
         tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(s_free);                               // S may be overwritten by the next Q K^T
         // boundary chunks (some of the warp's rows see only part of them) are masked in registers:
         // column c is allowed iff c_lo <= c < c_hi, one unsigned compare; chunks inside the
         // intersection of the warp's rows skip this
@@ -458,24 +445,25 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const bool need = m_t > m + 8.0f;
         const float m_new = need ? m_t : m;
         const float alpha = need ? fast_exp2(m - m_new) : 1.0f;
-        // O has to be rescaled only where something has been accumulated (l > 0); that is the one place where a
-        // warp waits for the P V of the previous key tile, i.e. for the other warps
-        if (__any_sync(0xffffffffu, need && l > 0.f)) {
-          const uint32_t pj = j - 1;                       // l > 0 implies j > 0
-          mbar_wait(&pv_done[pj % NSB], (pj / NSB) & 1, abort_flag, p.status, 0x1900);
+        const bool any_need = __any_sync(0xffffffffu, need);
+        if (j > 0) {
+          mbar_wait(pv_done, (j - 1) & 1, abort_flag, p.status, 0x1900);   // P buffer and O are free
           tc_fence_after();
+          if (any_need) {
 #pragma unroll
-          for (int c = 0; c < HD / 32; ++c) {
-            uint32_t orr[32];
-            tmem_ld32(lane_addr + O_COL + 32 * c, orr);
-            tc_wait_ld();
+            for (int c = 0; c < HD / 32; ++c) {
+              uint32_t orr[32];
+              tmem_ld32(lane_addr + O_COL + 32 * c, orr);
+              tc_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-            tmem_st32(lane_addr + O_COL + 32 * c, orr);
+              for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+              tmem_st32(lane_addr + O_COL + 32 * c, orr);
+            }
           }
         }
-        // p = 2^(s*scale - m) chunk by chunk, packed to bf16 pairs and written over the first half of this
-        // row's S (masked scores are -inf, so p = 0); two scores per packed fp32x2 multiply-add and add
+        // p = 2^(s*scale - m) chunk by chunk, packed to bf16 pairs and written to TMEM at once
+        // (masked scores are -inf, so p = 0)
+        // (two scores per packed fp32x2 multiply-add and per packed add)
         float2 rs_a = make_float2(0.f, 0.f), rs_b = make_float2(0.f, 0.f);
         const float2 sl2_2 = make_float2(sl2, sl2), nm_2 = make_float2(-m_new, -m_new);
 #pragma unroll
@@ -499,13 +487,13 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
             for (int i = 0; i < 16; ++i) pk[i] = 0u;
           }
-          tmem_st16(s_addr + 16 * c, pk);
+          tmem_st16(lane_addr_p + 16 * c, pk);
         }
         l = l * alpha + ((rs_a.x + rs_a.y) + (rs_b.x + rs_b.y));
         m = m_new;
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(&p_full[sbuf]);
+        mbar_arrive(p_full);
       }
     }
     // ---------------- epilogue: the global tokens join the softmax, then O / l
@@ -543,7 +531,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     for (int g = 0; g < G; ++g) l_f += fast_exp2(s_sg[g * 128 + row] - m_f);
     const float inv = 1.0f / l_f;
     if (j > 0) {
-      mbar_wait(&pv_done[(j - 1) % NSB], ((j - 1) / NSB) & 1, abort_flag, p.status, 0x1A00);
+      mbar_wait(pv_done, (j - 1) & 1, abort_flag, p.status, 0x1A00);
       tc_fence_after();
     }
     float of[HD];
@@ -623,7 +611,10 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (warp == 5) tmem_dealloc(tmem, TMEM_COLS);
+  if (warp == 5) {
+    tmem_dealloc(tmem, TMEM_COLS);
+    tmem_dealloc(tmem_p, TMEM_P_COLS);
+  }
 }
 
 // ------------------------------------------------------------------------------------------

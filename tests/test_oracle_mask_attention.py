@@ -171,3 +171,29 @@ def test_filtered_positions_match_masked_subset():
     mask[1:, 1:] = pm
     ref = _torch_masked_attention(q, k, v, mask, 0.25)
     assert np.abs(o - ref).max() < 2e-6
+
+
+def test_permutation_inside_blocks_leaves_attention_unchanged():
+    """The key set of Sec. 3.2 depends on a token's block only: presenting the tokens of every block in
+    another order (positions, Q, K and V permuted alike) permutes the output rows and nothing else; the
+    same holds for the order of whole blocks."""
+    h, w, b, r = 8, 12, 4, 1
+    rng = np.random.default_rng(8)
+    pos = np.arange(h * w, dtype=np.int32)
+    n = 1 + pos.size
+    q, k, v = synth.attention_qkv(12, 1, n, 2, 16)
+    base, bsc = oracle.attention(q, k, v, h, w, b, r, patch_pos=pos[None], want_scores=True)
+    blk = (pos // w) // b * (w // b) + (pos % w) // b
+    # shuffle inside blocks, then shuffle the blocks themselves
+    key = rng.permutation(blk.max() + 1)[blk] * 1000.0 + rng.random(pos.size)
+    perm = np.argsort(key)
+    assert not np.array_equal(perm, pos)
+
+    def reorder(a):
+        out = a.copy()
+        out[:, 1:] = a[:, 1 + perm]
+        return out
+    got, gsc = oracle.attention(reorder(q), reorder(k), reorder(v), h, w, b, r, patch_pos=pos[perm][None],
+                                want_scores=True)
+    assert np.abs(got - reorder(base)).max() < 1e-6
+    assert np.abs(gsc - bsc[:, :, perm]).max() < 1e-7

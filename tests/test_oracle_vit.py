@@ -21,6 +21,10 @@ def _torch_forward(arch, cfg, w, image, gh, gw, forced_keep=None):
     x = torch.cat([t(w["cls"])[None].expand(B, -1, -1), x], 1) + t(w["pos"])[None]
     pos = torch.arange(gh * gw)[None].expand(B, -1)
     kept = None
+    # filter stages written out here, independently of the oracle's helpers: (layer, keep ratio) pairs
+    stages = list(cfg.get("filters") or
+                  ([(cfg["filter_layer"], cfg["keep_ratio"])] if cfg.get("filter_layer", 0) > 0 else []))
+    kept_positions, taken = [], 0
     for li, lw in enumerate(w["layers"], start=1):
         N = x.shape[1]
         h = F.layer_norm(x, (D,), t(lw["ln1_g"]), t(lw["ln1_b"]), arch["ln_eps"])
@@ -46,11 +50,16 @@ def _torch_forward(arch, cfg, w, image, gh, gw, forced_keep=None):
             u = F.gelu(u)
         m = F.linear(u, t(lw["w_fc2"]), t(lw["b_fc2"]))
         x = x + (t(lw["ls2"]) * m if "ls2" in lw else m)
-        if li == cfg.get("filter_layer", 0):
+        for layer, ratio in stages:
+            if li != layer:
+                continue
             npatch = N - G
-            kk = int(np.ceil(cfg["keep_ratio"] * npatch - 1e-9))
+            kk = int(np.ceil(ratio * npatch - 1e-9))
             if forced_keep is not None:
-                kept = torch.from_numpy(np.asarray(forced_keep)).long()
+                # original positions of this stage's survivors -> indices among the tokens present
+                want = torch.from_numpy(np.asarray(forced_keep)[:, taken:taken + kk]).long()
+                kept = torch.stack([torch.searchsorted(pos[b].contiguous(), want[b]) for b in range(B)])
+                assert bool((torch.gather(pos, 1, kept) == want).all())
             else:
                 score = p[:, :, 0, G:].to(torch.float32).mean(1)
                 order = torch.argsort(-score.double(), dim=-1, stable=True)[:, :kk]
@@ -58,8 +67,10 @@ def _torch_forward(arch, cfg, w, image, gh, gw, forced_keep=None):
             idx = torch.cat([torch.arange(G)[None].expand(B, -1), kept + G], 1)
             x = torch.gather(x, 1, idx[:, :, None].expand(-1, -1, D))
             pos = torch.gather(pos, 1, kept)
+            kept_positions.append(pos.clone())
+            taken += kk
     out = F.layer_norm(x, (D,), t(w["lnf_g"]), t(w["lnf_b"]), arch["ln_eps"])
-    return out.numpy(), None if kept is None else kept.numpy()
+    return out.numpy(), None if not kept_positions else torch.cat(kept_positions, 1).numpy()
 
 
 def _setup(arch, gh, gw, seed=0, batch=2):
@@ -83,6 +94,49 @@ def test_forward_matches_library_restatement(gh, gw, kind, ls, G):
     if np.array_equal(wkept2, got["kept_idx"]):
         assert np.abs(got["out"] - want2).max() < 2e-5
     assert got["out"].shape == (2, G + oracle.keep_count(gh * gw, 0.6), 64)
+
+
+@pytest.mark.parametrize("gh,gw,kind,stages", [
+    (8, 8, synth.MLP_GELU, [(1, 0.6), (3, 0.5)]),
+    (9, 7, synth.MLP_SWIGLU, [(2, 0.75), (3, 0.4)]),
+    (10, 6, synth.MLP_GELU, [(1, 0.8), (2, 0.7), (4, 0.5)]),
+])
+def test_forward_with_several_filter_stages(gh, gw, kind, stages):
+    """Sec. 3.3 applied more than once: every stage ranks the tokens still present by that block's CLS
+    attention, survivors keep their original grid positions for the neighbourhood rule of Sec. 3.2."""
+    arch = synth.vit_tiny(layers=4, dim=64, heads=2, hidden=96, patch=4, mlp_kind=kind, layerscale=1)
+    w, img = _setup(arch, gh, gw, seed=11)
+    cfg = dict(arch, attn_mode=synth.ATTN_SPARSE, block=2, radius=1, filters=stages)
+    got = oracle.vit_forward(cfg, w, img, gh, gw)
+    counts, cur = [], gh * gw
+    for _, ratio in stages:
+        cur = int(np.ceil(ratio * cur - 1e-9))
+        counts.append(cur)
+    assert got["kept_all"].shape == (2, sum(counts)) and got["out"].shape == (2, 1 + counts[-1], 64)
+    # every stage's set is ascending, and a subset of the stage before
+    off, prev = 0, None
+    for c in counts:
+        seg = got["kept_all"][:, off:off + c]
+        assert (np.diff(seg, axis=1) > 0).all()
+        if prev is not None:
+            assert all(set(seg[b]) <= set(prev[b]) for b in range(2))
+        prev, off = seg, off + c
+    assert np.array_equal(got["kept_idx"], prev)
+    # teacher-forced with the oracle's own sets, the library restatement gives the same tokens
+    want, _ = _torch_forward(arch, cfg, w, img, gh, gw, forced_keep=got["kept_all"])
+    assert np.abs(got["out"] - want).max() < 2e-5
+    # and the oracle, forced with its own sets, reproduces itself exactly
+    again = oracle.vit_forward(cfg, w, img, gh, gw, forced_keep=got["kept_all"])
+    assert np.array_equal(again["out"], got["out"])
+    # free-running restatement: same sets unless two scores are closer than fp32 resolution
+    want2, wkept2 = _torch_forward(arch, cfg, w, img, gh, gw)
+    if np.array_equal(wkept2, got["kept_all"]):
+        assert np.abs(got["out"] - want2).max() < 2e-5
+    # one stage through the list form == the single-stage fields
+    one = oracle.vit_forward(dict(cfg, filters=stages[:1]), w, img, gh, gw)
+    legacy = dict(cfg, filter_layer=stages[0][0], keep_ratio=stages[0][1])
+    legacy.pop("filters")
+    assert np.array_equal(one["out"], oracle.vit_forward(legacy, w, img, gh, gw)["out"])
 
 
 def test_forward_dense_mode_and_structural_identities():
@@ -124,3 +178,9 @@ def test_building_blocks_against_library():
     for v in (-3.0, -0.5, 0.0, 0.7, 4.0):
         assert abs(oracle.gelu(v) - float(F.gelu(torch.tensor(v, dtype=torch.float64)))) < 1e-6
         assert abs(oracle.silu(v) - float(F.silu(torch.tensor(v, dtype=torch.float64)))) < 1e-6
+    # the array forms of the two activations (what the timed CPU baseline loops over)
+    a = rng.standard_normal(1000).astype(np.float32) * 3
+    g2 = rng.standard_normal(1000).astype(np.float32)
+    ta, tg = torch.from_numpy(a).double(), torch.from_numpy(g2).double()
+    assert np.abs(oracle.gelu_n(a) - F.gelu(ta).numpy()).max() < 1e-6
+    assert np.abs(oracle.silu_mul_n(a, g2) - (F.silu(ta) * tg).numpy()).max() < 2e-6
