@@ -33,10 +33,12 @@ constexpr int ATT_THREADS = 256;   // warps 0-3 softmax (one warpgroup), 4 TMA, 
                                    // warpgroup exists so that it can hand its registers to the first
 constexpr int TILE_BYTES = 128 * 128;  // Q tile
 constexpr int KV_BYTES = TK * 128;      // K or V tile
-constexpr int GROW_BYTES = 1024;   // global-token rows of one head: up to 8 x 128 B
-constexpr int ATT_SMEM = TILE_BYTES + 2 * KST * KV_BYTES + 2 * GROW_BYTES + 1024 /*align*/ + 256 /*barriers*/ +
-                         8 * 128 * 4 /*global-token scores*/;
-constexpr int MAXG = 8;
+constexpr int MAXG = 16;           // global tokens
+// Shared memory of a CTA for `grows` rows of global tokens (8 or 16: with up to 8, three CTAs fit an SM):
+// Q tile, K / V stages, the global tokens' key and value rows (128 B each), barriers, their scores per query row.
+constexpr int att_smem(int grows) {
+  return TILE_BYTES + 2 * KST * KV_BYTES + 2 * grows * 128 + 1024 /*align*/ + 256 /*barriers*/ + grows * 128 * 4;
+}
 // two TMEM allocations per CTA, 160 columns in all, so that three CTAs share an SM's 512
 constexpr uint32_t TMEM_COLS = 128, TMEM_P_COLS = 32;
 constexpr uint32_t S_COL = 0, O_COL = 64;
@@ -207,6 +209,7 @@ struct PatchParams {
   __nv_bfloat16* o;
   int64_t o_sb, o_st, o_sh;
   int nbx, nby, nb, radius, n_global, n_patch, tiles_per_image;
+  int grows;                       // rows reserved for the global tokens in shared memory (8 or 16)
   float scale_log2;
   uint32_t* status;
 };
@@ -250,8 +253,8 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   uint8_t* sK = smem + TILE_BYTES;
   uint8_t* sV = sK + KST * KV_BYTES;
   uint8_t* sKg = sV + KST * KV_BYTES;      // global-token key rows (G x 128 B, swizzled)
-  uint8_t* sVg = sKg + GROW_BYTES;                       // global-token value rows
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sVg + GROW_BYTES);
+  uint8_t* sVg = sKg + p.grows * 128;                    // global-token value rows
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sVg + p.grows * 128);
   uint64_t* q_full = bars;
   uint64_t* k_full = bars + 1;
   uint64_t* k_empty = k_full + KST;
@@ -871,10 +874,9 @@ int32_t spv_attn_plan_build(spv_ctx* ctx, int32_t batch, int32_t grid_h, int32_t
 }
 
 int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, cudaStream_t stream) {
-  static bool configured = false;
-  if (!configured) {
-    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM));
-    configured = true;
+  if (!ctx->attn_configured) {
+    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, att_smem(MAXG)));
+    ctx->attn_configured = 1;
   }
   const int n_tok = plan->n_global + plan->n_patch;
   CUtensorMap tq, tk, tv, tkg, tvg;
@@ -891,6 +893,7 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   pp.o = (__nv_bfloat16*)io->o; pp.o_sb = io->o_sb; pp.o_st = io->o_st; pp.o_sh = io->o_sh;
   pp.nbx = plan->nbx; pp.nby = plan->nby; pp.nb = plan->nb; pp.radius = plan->radius;
   pp.n_global = plan->n_global; pp.n_patch = plan->n_patch; pp.tiles_per_image = plan->tiles_per_image;
+  pp.grows = plan->n_global <= 8 ? 8 : MAXG;
   pp.scale_log2 = io->scale * 1.4426950408889634f;
   pp.status = ctx->d_status;
   const dim3 grid(plan->tiles_per_image, io->heads, plan->batch);
@@ -898,7 +901,7 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   // the output as a tensor map (same row order as Q, boxes of 32 rows): warps whose rows are all valid store by TMA
   CUtensorMap to;
   if ((st = make_qkv_map(ctx, &to, io->o, io->o_sb, io->o_st, io->o_sh, n_tok, io->heads, plan->batch, 32)) != SPV_OK) return st;
-  attn_patch_kernel<<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, tkg, tvg, to, pp);
+  attn_patch_kernel<<<grid, ATT_THREADS, att_smem(pp.grows), stream>>>(tq, tk, tv, tkg, tvg, to, pp);
   return spv_launch_ok(ctx);
 }
 

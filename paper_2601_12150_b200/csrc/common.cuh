@@ -26,6 +26,11 @@ struct spv_ctx {
   uint32_t last_site;            // site code read by the last failing spv_check
   struct SpvProf* prof;          // event record of spv_profile_enable (NULL until first enabled)
   int32_t prof_on;
+  // one-time per-device launch configuration (function attributes are per device, and a context is bound to one)
+  int32_t attn_configured;
+  int32_t gemm_single_configured[8];   // per epilogue variant
+  int32_t gemm_max_pairs[8];     // per epilogue variant: CTA pairs of the pair-form GEMM that can be resident at
+                                 // once (0 = not yet queried)
 };
 
 // Event pair around one launch group while profiling is on (no-ops otherwise).

@@ -387,7 +387,8 @@ int32_t launch(spv_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tw, const
   const int n_tiles = (d->n + BN - 1) / BN;
   if (use_pair(d)) {
     // pair form: clusters of two CTAs, as many as can be resident at once
-    static int max_pairs = 0;
+    static_assert(EPI >= 0 && EPI < 8, "per-context launch state is indexed by the epilogue variant");
+    int& max_pairs = ctx->gemm_max_pairs[EPI];
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -410,10 +411,9 @@ int32_t launch(spv_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tw, const
     SPV_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_bf16_kernel<EPI, true>, ta, tw, tout, d->m, d->n, d->k, ep, ctx->d_status));
     return spv_launch_ok(ctx);
   }
-  static bool configured = false;
-  if (!configured) {
+  if (!ctx->gemm_single_configured[EPI]) {
     SPV_CUDA_OK(cudaFuncSetAttribute(gemm_bf16_kernel<EPI, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
-    configured = true;
+    ctx->gemm_single_configured[EPI] = 1;
   }
   const int tiles = ((d->m + BM - 1) / BM) * n_tiles;
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;

@@ -192,7 +192,7 @@ int32_t vit_layout(const spv_vit_config* c, int32_t batch, int32_t gh, int32_t g
   if (c->layers < 1 || c->dim < 64 || c->heads < 1 || c->mlp_hidden < 8 || c->patch < 1) return SPV_ERR_INVALID_ARG;
   if (c->dim != c->heads * 64) return SPV_ERR_UNSUPPORTED;               // head_dim 64 only
   if (c->dim % 8 || c->mlp_hidden % 8) return SPV_ERR_ALIGNMENT;
-  if (c->n_global < 1 || c->n_global > 8) return SPV_ERR_UNSUPPORTED;
+  if (c->n_global < 1 || c->n_global > 16) return SPV_ERR_UNSUPPORTED;
   if (c->mlp_kind != SPV_MLP_GELU && c->mlp_kind != SPV_MLP_SWIGLU) return SPV_ERR_INVALID_ARG;
   if (c->attn_mode != SPV_ATTN_DENSE && c->attn_mode != SPV_ATTN_SPARSE) return SPV_ERR_INVALID_ARG;
   if (c->block < 1 || c->radius < 0) return SPV_ERR_INVALID_ARG;

@@ -1,6 +1,7 @@
 """GPU parity of spatial_block_attention (Sec. 3.2) against the CPU oracle on the same seeded
 bf16 inputs.  Tolerance for bf16 outputs vs the fp32/fp64 oracle: max |err| <= 2e-2 and
-relative L2 <= 5e-3."""
+relative L2 <= 5e-3.  CLS->patch scores (fp32 on both sides, Sec. 3.3 ranks by them): per (image, head)
+row max |err| <= 1e-2 * max(ref) and relative L2 <= 5e-3, at every size."""
 import numpy as np
 import pytest
 import torch
@@ -25,6 +26,33 @@ def _check(got, ref, max_abs=2e-2, rel_l2=5e-3):
     assert np.abs(err).max() <= max_abs, np.abs(err).max()
     rel = np.linalg.norm(err) / np.linalg.norm(ref)
     assert rel <= rel_l2, rel
+
+
+def _check_scores(got, ref):
+    """fp32 softmax weights of the CLS row, [B, h, n_patch]: relative bounds per (image, head) row, so that
+    the check means the same at 196 and at 21,316 patch columns (where a weight is about 5e-5)."""
+    assert got.shape == ref.shape
+    assert np.isfinite(got).all()
+    g = got.astype(np.float64).reshape(-1, got.shape[-1])
+    w = ref.astype(np.float64).reshape(-1, ref.shape[-1])
+    err = np.abs(g - w).max(axis=1)
+    assert (err <= 1e-2 * w.max(axis=1)).all(), (err / w.max(axis=1)).max()
+    rel = np.linalg.norm(g - w, axis=1) / np.linalg.norm(w, axis=1)
+    assert (rel <= 5e-3).all(), rel.max()
+
+
+def _check_topk_of_mean(got, ref, keep=0.5):
+    """The kept set of Sec. 3.3 from the GPU's scores equals the one from the oracle's scores, apart from
+    tokens whose oracle mean lies within 1e-3 relative of the oracle's threshold."""
+    for b in range(ref.shape[0]):
+        mg, mw = got[b].astype(np.float64).mean(axis=0), ref[b].astype(np.float64).mean(axis=0)
+        k = int(np.ceil(keep * mw.size - 1e-9))
+        kept_g = set(np.argsort(-mg, kind="stable")[:k].tolist())
+        order_w = np.argsort(-mw, kind="stable")
+        kept_w = set(order_w[:k].tolist())
+        thr = mw[order_w[k - 1]]
+        for t in kept_g ^ kept_w:
+            assert abs(mw[t] - thr) <= 1e-3 * abs(thr), (t, mw[t], thr)
 
 
 def _to_dev(ctx, a, packed=False):
@@ -52,7 +80,7 @@ def test_single_attention_op_28x28(ctx):
     want, wsc = oracle.attention(q, k, v, 28, 28, 7, 1, want_scores=True)
     got, gsc = _run(ctx, q, k, v, 28, 28, 7, 1)
     _check(got, want)
-    assert np.abs(gsc - wsc).max() < 2e-4 * max(1.0, wsc.max() / 1e-2)
+    _check_scores(gsc, wsc)
     dense = oracle.dense_attention(q, k, v)
     got3, _ = _run(ctx, q, k, v, 28, 28, 7, 3)
     _check(got3, dense)
@@ -68,7 +96,9 @@ def test_single_attention_op_28x28(ctx):
     (20, 20, 16, 0, 1, 1, 2),     # blocks larger than a tile (256 tokens), own block only
     (9, 30, 4, 3, 1, 2, 1),       # wide neighbourhood
     (12, 12, 1, 1, 1, 1, 2),      # one patch per block: 3x3-patch windows, a query tile per grid row
-    (10, 14, 3, 0, 8, 1, 1),      # own block only, the maximum of eight global tokens
+    (10, 14, 3, 0, 8, 1, 1),      # own block only, eight global tokens (the most that leave three CTAs per SM)
+    (18, 11, 8, 1, 9, 1, 2),      # nine global tokens (CLS + eight registers)
+    (16, 24, 8, 1, 16, 2, 1),     # the maximum of sixteen global tokens
     (5, 3, 8, 1, 1, 1, 1),        # a grid smaller than one block
 ])
 def test_geometries(ctx, gh, gw, b, r, G, B, H):
@@ -77,7 +107,7 @@ def test_geometries(ctx, gh, gw, b, r, G, B, H):
     want, wsc = oracle.attention(q, k, v, gh, gw, b, r, n_global=G, want_scores=True)
     got, gsc = _run(ctx, q, k, v, gh, gw, b, r, G=G, packed=True)
     _check(got, want)
-    assert np.abs(gsc - wsc).max() < 1e-3
+    _check_scores(gsc, wsc)
 
 
 def test_filtered_tokens_row_major_and_block_major(ctx):
@@ -95,7 +125,7 @@ def test_filtered_tokens_row_major_and_block_major(ctx):
     want, wsc = oracle.attention(q, k, v, gh, gw, b, r, patch_pos=keep, want_scores=True)
     got, gsc = _run(ctx, q, k, v, gh, gw, b, r, patch_pos=keep)
     _check(got, want)
-    assert np.abs(gsc - wsc).max() < 1e-3
+    _check_scores(gsc, wsc)
     # same tokens presented in block-major order
     perm = np.stack([np.lexsort((keep[i], (keep[i] % gw) // b, (keep[i] // gw) // b)) for i in range(B)])
     def reorder(a):
@@ -107,7 +137,7 @@ def test_filtered_tokens_row_major_and_block_major(ctx):
     got_bm, gsc_bm = _run(ctx, reorder(q), reorder(k), reorder(v), gh, gw, b, r, patch_pos=keep_bm, order=1)
     _check(got_bm, reorder(want))
     for i in range(B):
-        assert np.abs(gsc_bm[i] - wsc[i][:, perm[i]]).max() < 1e-3
+        _check_scores(gsc_bm[i], wsc[i][:, perm[i]])
 
 
 def test_full_grid_block_major(ctx):
@@ -149,7 +179,8 @@ def test_sampled_rows_at_full_size(ctx):
     rows = np.unique(np.concatenate([[0, 1, gh * gw], rng.integers(1, 1 + gh * gw, size=300)])).astype(np.int32)
     want, wsc = oracle.attention(q, k, v, gh, gw, 8, 1, rows=rows, want_scores=True)
     _check(got[:, rows], want[:, rows])
-    assert np.abs(gsc - wsc).max() < 1e-3
+    _check_scores(gsc, wsc)
+    _check_topk_of_mean(gsc, wsc)
 
 
 def test_sampled_rows_146_grid_radius_2(ctx):
@@ -163,7 +194,8 @@ def test_sampled_rows_146_grid_radius_2(ctx):
     rows = np.unique(np.concatenate([[0, 1, gh * gw], edge, rng.integers(1, 1 + gh * gw, size=200)])).astype(np.int32)
     want, wsc = oracle.attention(q, k, v, gh, gw, 8, 2, rows=rows, want_scores=True)
     _check(got[:, rows], want[:, rows])
-    assert np.abs(gsc - wsc).max() < 1e-3
+    _check_scores(gsc, wsc)
+    _check_topk_of_mean(gsc, wsc)
 
 
 def test_sampled_rows_filtered_full_size(ctx):
@@ -203,7 +235,7 @@ def test_random_geometries_both_token_orders(ctx, seed):
     gh, gw = int(rng.integers(3, 48)), int(rng.integers(3, 48))
     b = int(rng.choice([1, 2, 3, 4, 7, 8, 16]))
     r = int(rng.choice([0, 1, 1, 2, 3]))
-    G = int(rng.choice([1, 1, 2, 8]))
+    G = int(rng.choice([1, 1, 2, 5, 9, 16]))
     B, H = int(rng.integers(1, 3)), int(rng.integers(1, 4))
     keep = rng.choice([0.0, 0.0, 0.3, 0.5, 0.9])
     n0 = gh * gw
@@ -220,7 +252,7 @@ def test_random_geometries_both_token_orders(ctx, seed):
                                  want_scores=True)
     got, gsc = _run(ctx, q, k, v, gh, gw, b, r, G=G, patch_pos=pos if have_pos else None)
     _check(got, want)
-    assert np.abs(gsc - wsc).max() < 1e-3
+    _check_scores(gsc, wsc)
     perm = np.stack([np.lexsort((pos[i], (pos[i] % gw) // b, (pos[i] // gw) // b)) for i in range(B)])
 
     def reorder(a):
@@ -232,4 +264,4 @@ def test_random_geometries_both_token_orders(ctx, seed):
     got_bm, gsc_bm = _run(ctx, reorder(q), reorder(k), reorder(v), gh, gw, b, r, G=G, patch_pos=pos_bm, order=1)
     _check(got_bm, reorder(want))
     for i in range(B):
-        assert np.abs(gsc_bm[i] - wsc[i][:, perm[i]]).max() < 1e-3
+        _check_scores(gsc_bm[i], wsc[i][:, perm[i]])
