@@ -472,6 +472,384 @@ def run_gpu(args, wl, rank, world):
         dist.destroy_process_group()
 
 
+
+# --------------------------------------------------------------------------------------------
+# single-operation workloads: the hot-path kernels timed alone through the C ABI
+# --------------------------------------------------------------------------------------------
+def coherent_kept(seed, grid, keep):
+    """A spatially coherent kept set (what Sec. 3.3 leaves on a real slide: background goes, tissue stays):
+    the complement of a low-frequency background mask, exactly ceil(keep * grid^2) positions, ascending."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    n = grid * grid
+    k = int(np.ceil(keep * n - 1e-9))
+    bg = synth.background_mask(rng, grid, grid, 1.0 - k / n).reshape(-1)
+    kept = np.flatnonzero(~bg)[:k]
+    if kept.size < k:
+        kept = np.sort(np.concatenate([kept, np.flatnonzero(bg)[:k - kept.size]]))
+    return kept.astype(np.int32)
+
+
+def block_major(pos, grid, block):
+    """Positions reordered by (block row, block column, position): the order vit_forward keeps internally."""
+    return pos[np.lexsort((pos, (pos % grid) // block, (pos // grid) // block))]
+
+
+OP_WORKLOADS = {
+    # attention: (grid, block, radius, batch, heads, kept, pattern)
+    "attn_28x28_b1": ("attn", dict(grid=28, block=7, radius=1, batch=1, heads=16)),
+    "attn_28x28_b64": ("attn", dict(grid=28, block=7, radius=1, batch=64, heads=16)),
+    "attn_128x128_b4_r1": ("attn", dict(grid=128, block=8, radius=1, batch=4, heads=16)),
+    "attn_128x128_b4_r2": ("attn", dict(grid=128, block=8, radius=2, batch=4, heads=16)),
+    "attn_128x128_b4_r3": ("attn", dict(grid=128, block=8, radius=3, batch=4, heads=16)),
+    "attn_128x128_b2_dense": ("attn", dict(grid=128, block=8, radius=16, batch=2, heads=16)),
+    "attn_128x128_b4_keep50_scattered": ("attn", dict(grid=128, block=8, radius=1, batch=4, heads=16, keep=0.5,
+                                                      pattern="scattered")),
+    "attn_128x128_b4_keep50_coherent": ("attn", dict(grid=128, block=8, radius=1, batch=4, heads=16, keep=0.5,
+                                                     pattern="coherent")),
+    # filter: (grid, batch, heads, dim, keep, cold L2)
+    "filter_64x64_b1": ("filter", dict(grid=64, batch=1, heads=16, dim=1024, keep=0.5, cold=False)),
+    "filter_64x64_b1_cold": ("filter", dict(grid=64, batch=1, heads=16, dim=1024, keep=0.5, cold=True)),
+    "filter_256x256_b4": ("filter", dict(grid=256, batch=4, heads=16, dim=1024, keep=0.5, cold=False)),
+    # GEMMs of one ViT-L/16 block at 2048x2048, batch 4 (M = 4 * 16385 rows)
+    "gemm_qkv_65540": ("gemm", dict(m=65540, n=3072, k=1024, epi="bias")),
+    "gemm_out_65540": ("gemm", dict(m=65540, n=1024, k=1024, epi="resid")),
+    "gemm_fc1_65540": ("gemm", dict(m=65540, n=4096, k=1024, epi="gelu")),
+    "gemm_fc2_65540": ("gemm", dict(m=65540, n=1024, k=4096, epi="resid")),
+    # LayerNorm at the full and post-filter row counts
+    "ln_65540x1024": ("ln", dict(rows=65540, dim=1024)),
+    "ln_32772x1024": ("ln", dict(rows=32772, dim=1024)),
+}
+
+
+def time_op(torch, fn, iters, flush=None):
+    """Mean device time of fn() in ms over `iters` calls (CUDA events on the current stream, after three
+    warm-up calls).  With `flush` (a buffer larger than L2) every call is preceded by a write of that buffer
+    and timed by its own event pair, so that the operands come from HBM."""
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+    tot = 0.0
+    for _ in range(iters):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        tot += e0.elapsed_time(e1)
+    return tot / iters
+
+
+def run_op(args, name):
+    """One JSON line for a single-operation workload: the rate in the roofline's unit, the roofline object
+    (useful FLOP or algorithmic bytes / CUDA-event time / measured peak) and the oracle timed on the same
+    operation (a bounded sample of it)."""
+    import torch
+    import oracle
+    import paper_2601_12150_b200 as spv
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = spv.Context(0)
+    pk = peaks()
+    kind, o = OP_WORKLOADS[name]
+    iters = max(args.steps, 1) * 5
+    launches0 = ctx.launch_count()
+    cfg = {"workload": name}
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    sampler.start()
+    if kind == "attn":
+        g, b, r, B, H = o["grid"], o["block"], o["radius"], o["batch"], o["heads"]
+        pos_dev, pos_host, order = None, None, spv.TOKENS_ROW_MAJOR
+        if "keep" in o:
+            rows = []
+            for i in range(B):
+                if o["pattern"] == "scattered":
+                    rng = np.random.Generator(np.random.PCG64(100 + i))
+                    kept = np.sort(rng.choice(g * g, size=int(np.ceil(o["keep"] * g * g - 1e-9)), replace=False)).astype(np.int32)
+                else:
+                    kept = coherent_kept(200 + i, g, o["keep"])
+                rows.append(block_major(kept, g, b))
+            pos_host = np.stack(rows)
+            pos_dev = torch.from_numpy(pos_host).to(dev)
+            order = spv.TOKENS_BLOCK_MAJOR
+            n_patch = pos_host.shape[1]
+        else:
+            n_patch = g * g
+            if g >= 64:          # the layout vit_forward uses: block-major tokens inside the fused QKV buffer
+                order = spv.TOKENS_BLOCK_MAJOR
+                pos_host = np.stack([block_major(np.arange(g * g, dtype=np.int32), g, b)] * B)
+                pos_dev = torch.from_numpy(pos_host).to(dev)
+        n = 1 + n_patch
+        gen = torch.Generator(device=dev).manual_seed(1)
+        qkv = torch.randn((B, n, 3, H, 64), device=dev, generator=gen).to(torch.bfloat16)
+        q, k, v = qkv[:, :, 0], qkv[:, :, 1], qkv[:, :, 2]
+        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=dev)
+        ctx.spatial_block_attention(q, k, v, g, g, b, r, patch_pos=pos_dev, token_order=order, want_scores=False, out=out)
+        ctx.check()
+        ctx.profile(True)
+        for _ in range(iters):
+            ctx.spatial_block_attention(q, k, v, g, g, b, r, patch_pos=pos_dev, token_order=order, want_scores=False, out=out)
+        prof = ctx.profile_read()
+        ctx.profile(False)
+        ctx.check()
+        ms_patch = prof["attn_patch"]["ms"] / iters
+        ms_all = sum(p_["ms"] for p_ in prof.values()) / iters
+        pairs = sum(attention_pairs(g, g, b, r, 1, None if pos_host is None else pos_host[i])[0] for i in range(B))
+        flop = 4.0 * 64 * H * pairs
+        achieved = flop / (ms_patch * 1e-3) / 1e12
+        cfg.update(grid=f"{g}x{g}", block=b, radius=r, batch=B, heads=H, tokens=n,
+                   token_order="block-major" if order == spv.TOKENS_BLOCK_MAJOR else "row-major",
+                   l2="inputs larger than L2" if qkv.numel() * 2 > 126e6 else "warm L2 (Q, K, V fit in L2)",
+                   ms_patch_kernel=ms_patch, ms_whole_call=ms_all,
+                   mean_tokens_per_block=n_patch / (-(-g // b)) ** 2)
+        value, unit = achieved, "useful TFLOP/s (patch-query kernel)"
+        roof = dict(kernel="attn_patch_kernel", bound="tensor", achieved=achieved, peak=pk["tensor_burst"], unit="TFLOP/s",
+                    frac=achieved / pk["tensor_burst"], traffic=None,
+                    peak_source=f"of {pk['source']} (burst bf16 figure: the kernel is timed alone)",
+                    frac_of_sustained=achieved / pk["tensor"])
+        # oracle: sampled query rows of image 0
+        nrow = min(n, 256 if n > 4096 else 785)
+        qh, kh, vh = (x_[:1].float().cpu().numpy() for x_ in (q, k, v))
+        rows = np.unique(np.linspace(0, n - 1, nrow).astype(np.int32))
+        t0 = time.perf_counter()
+        oracle.attention(qh, kh, vh, g, g, b, r, patch_pos=None if pos_host is None else pos_host[:1], rows=rows)
+        dt = time.perf_counter() - t0
+        cpu_rate = (flop / B) * (rows.size / n) / dt / 1e12
+        cpu = dict(value=cpu_rate, unit="useful TFLOP/s", cores=oracle.num_threads(), kind="oracle",
+                   sample=f"{rows.size} query rows of image 0, all heads ({dt:.1f} s)")
+    elif kind == "filter":
+        g, B, H, D, keep = o["grid"], o["batch"], o["heads"], o["dim"], o["keep"]
+        NP = g * g
+        sc_h = synth.filter_scores(1, B, H, g, g)
+        tok_h = synth.token_rows(1, B, 1 + NP, D) if B * NP <= 65536 else None      # uint16 bf16 bit patterns
+        sc = torch.from_numpy(sc_h).to(dev)
+        if tok_h is not None:
+            tok = torch.from_numpy(tok_h.view(np.int16)).to(dev).view(torch.bfloat16)
+        else:
+            tok = torch.randn((B, 1 + NP, D), device=dev, generator=torch.Generator(device=dev).manual_seed(2)).to(torch.bfloat16)
+        kk = spv.filter_keep_count(NP, keep)
+        out = torch.empty((B, 1 + kk, D), dtype=torch.bfloat16, device=dev)
+        kept = torch.empty((B, kk), dtype=torch.int32, device=dev)
+        fn = lambda: ctx.cls_score_topk_filter(sc, tok, 1, keep, tokens_out=out, kept_idx=kept)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if o["cold"] else None
+        ms = time_op(torch, fn, iters, flush)
+        ctx.check()
+        ctx.profile(True)
+        for _ in range(iters):
+            if flush is not None:
+                flush.zero_()
+            fn()
+        prof = ctx.profile_read()
+        ctx.profile(False)
+        nbytes = B * (H * NP * 4 + 2 * (1 + kk) * D * 2 + kk * 4)
+        achieved = nbytes / (ms * 1e-3) / 1e9
+        gather_gbs = prof["filter_gather"]["work"] / (prof["filter_gather"]["ms"] * 1e-3) / 1e9
+        cfg.update(grid=f"{g}x{g}", batch=B, heads=H, dim=D, keep_ratio=keep, kept=kk, algorithmic_bytes=nbytes,
+                   l2=("L2 flushed before every call (256 MB written)" if o["cold"] else
+                       ("inputs larger than L2" if nbytes > 126e6 else "warm L2 (the operands fit in L2)")),
+                   ms_select=prof["filter_select"]["ms"] / iters, ms_gather=prof["filter_gather"]["ms"] / iters,
+                   gather_gbs=gather_gbs)
+        value, unit = achieved, "GB/s (whole call: head mean + select + gather)"
+        roof = dict(kernel="filter_gather", bound="hbm", achieved=gather_gbs, peak=pk["hbm"], unit="GB/s",
+                    frac=gather_gbs / pk["hbm"], traffic=None, peak_source=f"of {pk['source']}")
+        t0 = time.perf_counter()
+        oracle.token_filter(sc_h[:1], None if tok_h is None else tok_h[:1], n_global=1, keep_ratio=keep)
+        dt = time.perf_counter() - t0
+        per_img = nbytes / B if tok_h is not None else H * NP * 4 + kk * 4
+        cpu = dict(value=per_img / dt / 1e9, unit="GB/s", cores=oracle.num_threads(), kind="oracle",
+                   sample=f"image 0 ({'ranking and row gather' if tok_h is not None else 'ranking only'}, {dt:.2f} s)")
+    elif kind == "gemm":
+        M, N, K = o["m"], o["n"], o["k"]
+        gen = torch.Generator(device=dev).manual_seed(3)
+        a = (torch.randn((M, K), device=dev, generator=gen)).to(torch.bfloat16)
+        w = (torch.randn((N, K), device=dev, generator=gen) * 0.02).to(torch.bfloat16)
+        bias = torch.randn(N, device=dev, generator=gen)
+        if o["epi"] == "resid":
+            outb = torch.zeros((M, N), dtype=torch.float32, device=dev)
+            scale = torch.full((N,), 0.1, device=dev)
+            fn = lambda: ctx.gemm_bf16(a, w, outb, spv.EPI_BIAS_SCALE_RESID, bias=bias, scale=scale)
+            out_bytes = M * N * 4 * 2
+        else:
+            outb = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            epi = spv.EPI_BIAS_GELU if o["epi"] == "gelu" else spv.EPI_BIAS
+            fn = lambda: ctx.gemm_bf16(a, w, outb, epi, bias=bias)
+            out_bytes = M * N * 2
+        ms = time_op(torch, fn, iters)
+        ctx.check()
+        flop = 2.0 * M * N * K
+        achieved = flop / (ms * 1e-3) / 1e12
+        cfg.update(m=M, n=N, k=K, epilogue=o["epi"], l2="operands and output larger than L2",
+                   algorithmic_bytes=2 * (M * K + N * K) + out_bytes)
+        value, unit = achieved, "TFLOP/s"
+        roof = dict(kernel="gemm_bf16_kernel", bound="tensor", achieved=achieved, peak=pk["tensor_burst"], unit="TFLOP/s",
+                    frac=achieved / pk["tensor_burst"], traffic=None,
+                    peak_source=f"of {pk['source']} (burst bf16 figure: the kernel is timed alone)",
+                    frac_of_sustained=achieved / pk["tensor"])
+        rows = 256
+        ah = a[:rows].float().cpu().numpy()
+        wh = w.float().cpu().numpy()
+        oracle.linear(ah[:8], wh, None)
+        t0 = time.perf_counter()
+        oracle.linear(ah, wh, bias.cpu().numpy())
+        dt = time.perf_counter() - t0
+        cpu = dict(value=2.0 * rows * N * K / dt / 1e12, unit="TFLOP/s", cores=oracle.num_threads(), kind="oracle",
+                   sample=f"{rows} rows of A against the whole weight ({dt:.2f} s), without the activation")
+    else:
+        R, D = o["rows"], o["dim"]
+        gen = torch.Generator(device=dev).manual_seed(4)
+        x = torch.randn((R, D), device=dev, generator=gen)
+        gam = torch.randn(D, device=dev, generator=gen)
+        bet = torch.randn(D, device=dev, generator=gen)
+        y = torch.empty((R, D), dtype=torch.bfloat16, device=dev)
+        fn = lambda: ctx.layernorm(x, gam, bet, 1e-6, out=y)
+        ms = time_op(torch, fn, iters)
+        ctx.check()
+        nbytes = R * D * 6
+        achieved = nbytes / (ms * 1e-3) / 1e9
+        cfg.update(rows=R, dim=D, algorithmic_bytes=nbytes, l2="input + output larger than L2")
+        value, unit = achieved, "GB/s"
+        roof = dict(kernel="layernorm_kernel", bound="hbm", achieved=achieved, peak=pk["hbm"], unit="GB/s",
+                    frac=achieved / pk["hbm"], traffic=None, peak_source=f"of {pk['source']}")
+        rows = min(R, 16384)
+        xh = x[:rows].cpu().numpy()
+        t0 = time.perf_counter()
+        oracle.layernorm(xh, gam.cpu().numpy(), bet.cpu().numpy(), 1e-6)
+        dt = time.perf_counter() - t0
+        cpu = dict(value=rows * D * 6 / dt / 1e9, unit="GB/s", cores=oracle.num_threads(), kind="oracle",
+                   sample=f"{rows} rows ({dt:.2f} s)")
+    clocks = sampler.stop()
+    print(json.dumps({"metric": name, "value": value, "unit": unit, "n_gpus": 1, "steps": iters, "warmup": 3,
+                      "higher_is_better": True, "dtype": "bf16", "data": "synthetic", "config": cfg, "clocks": clocks,
+                      "gpu_launches": ctx.launch_count() - launches0, "roofline": roof, "cpu_baseline": cpu}))
+
+
+def run_microbench(args):
+    """The hardware rates the attention kernel's design is argued from, one JSON line per probe."""
+    import torch
+    import paper_2601_12150_b200 as spv
+    torch.cuda.set_device(0)
+    ctx = spv.Context(0)
+
+    def emit(name, r, unit, **extra):
+        sm = r["sm_count"]
+        print(json.dumps(dict(probe=name, per_clk_per_sm=r["units"] / r["cycles"] / sm, unit=unit + " / clk / SM",
+                              per_second=r["units"] / (r["ms"] * 1e-3), sm_mhz=r["cycles"] / r["ms"] / 1e3,
+                              ms=r["ms"], **extra)), flush=True)
+    for cps, thr in ((1, 128), (1, 512), (2, 1024)):
+        emit(f"ex2 ctas/SM={cps} threads={thr}", ctx.microbench("ex2", ctas_per_sm=cps, threads=thr, iters=4000), "ex2")
+    for poly in (0, 2, 4):
+        for cps, thr in ((2, 128), (3, 128), (2, 256)):
+            emit(f"softmax_body poly={poly}/8 ctas/SM={cps} threads={thr}",
+                 ctx.microbench("softmax_body", ctas_per_sm=cps, threads=thr, iters=500, poly_per_8=poly), "score")
+    for kind in ("mma_ss", "mma_ts"):
+        for m, n in ((128, 64), (64, 64), (128, 128), (128, 256)):
+            for iss in (1, 2, 4):
+                if iss * n + 32 > 512:
+                    continue
+                r = ctx.microbench(kind, m=m, n=n, iters=2000, issuers=iss)
+                emit(f"{kind} m={m} n={n} k=16 issuing warps={iss}", r, "FLOP",
+                     cycles_per_instruction_per_issuer=r["cycles"] / 8000)
+    for cps in (1, 2):
+        for rows, st in ((64, 4), (128, 4), (256, 2)):
+            emit(f"l2_tma ctas/SM={cps} box={rows}x128B stages={st}",
+                 ctx.microbench("l2_tma", ctas_per_sm=cps, box_rows=rows, stages=st, iters=4000), "byte")
+    ctx.check()
+
+
+# --------------------------------------------------------------------------------------------
+# ablation axes of the paper (Tables 2, 3, 5) as throughput sweeps: pruning ratio, window (block) size,
+# neighbourhood radius, number of global tokens, and filtering in two stages
+# --------------------------------------------------------------------------------------------
+def run_ablation(args):
+    """ViT-L/16 at 2048x2048, batch 4, one factor varied at a time around (block 8, radius 1, keep 0.5 after
+    block 4, one global token).  One JSON line per point: images/s, time and useful TFLOP/s of the patch-query
+    attention kernel, and the mean number of surviving tokens per spatial block after the filter."""
+    import torch
+    import paper_2601_12150_b200 as spv
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = spv.Context(0)
+    pk = peaks()
+    side, B = args.ablation_side, 4
+    base_arch = synth.vit_l16()
+    g = side // base_arch["patch"]
+    img = torch.from_numpy(synth.tissue_batch(6, B, side, side, background_range=(0.3, 0.6))).to(dev)
+    points = [("keep_ratio", kr, dict(keep=kr)) for kr in (0.6, 0.5, 0.4, 0.3, 0.2)]
+    points += [("block", b, dict(block=b)) for b in (2, 8, 16, 64)]
+    points += [("radius", r, dict(radius=r)) for r in (0, 1, 2, 3)]
+    points += [("n_global", G, dict(G=G)) for G in (1, 5, 9)]
+    points += [("filters", "4:0.7,12:0.7", dict(filters=[(4, 0.7), (12, 0.7)])),
+               ("filters", "4:0.5", dict(filters=[(4, 0.5)]))]
+    weights = {}
+    for axis, val, o in points:
+        G = o.get("G", 1)
+        arch = dict(base_arch, n_global=G)
+        if G not in weights:
+            weights.clear()
+            torch.cuda.empty_cache()
+            weights[G] = ctx.make_vit_weights(synth.vit_weights(2, arch, g, g))
+        dw = weights[G]
+        stages = o.get("filters", [(4, o.get("keep", 0.5))])
+        cfg = dict(arch, attn_mode=synth.ATTN_SPARSE, block=o.get("block", 8), radius=o.get("radius", 1), filters=stages)
+        wl = dict(name="ablation", arch=arch, cfg=dict(cfg, filter_layer=stages[0][0], keep_ratio=stages[0][1]),
+                  side=side, grid=g, batch=B)
+        kept = None
+        for _ in range(2):
+            _, kept = ctx.vit_forward(cfg, dw, img, g, g)
+        ctx.check()
+        steps = max(1, args.steps // 2)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            ctx.vit_forward(cfg, dw, img, g, g)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        ctx.profile(True)
+        for _ in range(steps):
+            ctx.vit_forward(cfg, dw, img, g, g)
+        prof = ctx.profile_read()
+        ctx.profile(False)
+        ctx.check()
+        kept_h = kept.cpu().numpy()
+        # useful attention FLOP of one step: stage boundaries split the layers
+        counts, cur = [], g * g
+        for _, ratio in stages:
+            cur = spv.filter_keep_count(cur, ratio)
+            counts.append(cur)
+        H = arch["heads"]
+        flop, prev_layer, off = 0.0, 0, 0
+        pos_sets = [None]
+        for c in counts:
+            pos_sets.append([kept_h[b, off:off + c] for b in range(B)])
+            off += c
+        bounds = [l for l, _ in stages] + [arch["layers"]]
+        for si, upto in enumerate(bounds):
+            n_layers = upto - prev_layer
+            prev_layer = upto
+            for b in range(B):
+                pp, _ = attention_pairs(g, g, cfg["block"], cfg["radius"], G, None if pos_sets[si] is None else pos_sets[si][b])
+                flop += n_layers * 4.0 * 64 * H * pp
+        nblocks = (-(-g // cfg["block"])) ** 2
+        attn_ms = prof["attn_patch"]["ms"] / steps
+        print(json.dumps({"axis": axis, "value": val, "image": f"{side}x{side}", "batch": B, "block": cfg["block"],
+                          "radius": cfg["radius"], "n_global": G, "filters": stages, "kept_final": counts[-1],
+                          "mean_survivors_per_block": counts[-1] / nblocks, "ms_per_step": ms,
+                          "images_per_s": B / (ms * 1e-3), "attn_patch_ms_per_step": attn_ms,
+                          "attn_useful_tflops": flop / (attn_ms * 1e-3) / 1e12,
+                          "attn_frac_of_sustained_bf16": flop / (attn_ms * 1e-3) / 1e12 / pk["tensor"],
+                          "gemm_ms_per_step": prof["gemm"]["ms"] / steps, "steps": steps}), flush=True)
+
+
 # --------------------------------------------------------------------------------------------
 # resolution sweep (ViT-L/16, batch 4): dense attention, neighbour-block sparse, sparse + filter
 # --------------------------------------------------------------------------------------------
@@ -532,7 +910,11 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS) + sorted(OP_WORKLOADS))
+    ap.add_argument("--microbench", action="store_true", help="hardware rate probes, one JSON line each")
+    ap.add_argument("--sweep-ablation", action="store_true",
+                    help="keep ratio / block / radius / global tokens / two filter stages, one JSON line per point")
+    ap.add_argument("--ablation-side", type=int, default=2048)
     ap.add_argument("--cpu-rows", type=int, default=16384, help="rows of the CPU-oracle sample")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--quick", action="store_true",
@@ -544,8 +926,22 @@ def main():
     if args.sweep:
         run_sweep(args)
         return
+    if args.microbench:
+        run_microbench(args)
+        return
+    if args.sweep_ablation:
+        run_ablation(args)
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus != world:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE is {world}: launch N > 1 with "
+                         "python -m torch.distributed.run --nproc-per-node N bench.py --gpus N")
+    if args.workload in OP_WORKLOADS:
+        if args.impl == "reference" or world > 1:
+            raise SystemExit("single-operation workloads run on one GPU with --impl ours")
+        run_op(args, args.workload)
+        return
     wl = workload_config(args.workload)
     if args.impl == "reference":
         run_reference(args, wl, rank)

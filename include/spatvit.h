@@ -58,6 +58,11 @@ int32_t spv_check(spv_ctx* ctx, void* stream);
 /* Site code of the bounded wait that the last failing spv_check() reported (0 = none): the
  * kernel and barrier that gave up, for diagnosis. */
 uint32_t spv_last_wait_site(const spv_ctx* ctx);
+/* Self-test of the bounded-wait path (no counterpart in the paper): launches one CTA in which one
+ * thread waits on a barrier that nobody arrives on.  The wait gives up after limit_ns (clamped to
+ * 1 ms), latches site code 0x5E1F and the kernel returns; the next spv_check() on the stream
+ * returns SPV_ERR_TIMEOUT, spv_last_wait_site() 0x5E1F, and the context stays usable. */
+int32_t spv_selftest_wait(spv_ctx* ctx, uint32_t limit_ns, void* stream);
 /* Number of kernels this context has launched so far (host counter, for accounting). */
 int64_t spv_launch_count(const spv_ctx* ctx);
 
@@ -81,7 +86,10 @@ typedef struct {
   float softmax_scale;           /* 0 => 1/sqrt(head_dim)                                       */
   int32_t n_patch;               /* patch tokens present per image (== H*W when patch_pos NULL) */
   const int32_t* patch_pos;      /* device [batch, n_patch] original positions y*W+x, each
-                                    position at most once per image; NULL = the full grid       */
+                                    position at most once per image, in the order token_order
+                                    states (checked on the device: a violation is latched, the
+                                    patch rows of o are then not written, and spv_check()
+                                    reports SPV_ERR_INVALID_ARG and clears it); NULL = full grid */
   int32_t token_order;           /* SPV_TOKENS_ROW_MAJOR: patch tokens in ascending position.
                                     SPV_TOKENS_BLOCK_MAJOR: patch tokens sorted by (block row,
                                     block column, position); avoids the internal regrouping copy */
@@ -157,7 +165,9 @@ int32_t cls_score_topk_filter(spv_ctx* ctx, const spv_filter_desc* desc, const f
  *     whose kernels can overlap on the GPU (different streams without an ordering) race on it:
  *     order them;
  *   - the call itself performs no cudaMalloc, cudaFree or other allocating routine; inputs and
- *     outputs are the caller's, exactly as for cls_score_topk_filter.  Asynchronous on `stream`. */
+ *     outputs are the caller's, exactly as for cls_score_topk_filter.  Asynchronous on `stream`;
+ *   - having no context, its launches appear neither in spv_launch_count() nor in the per-class
+ *     timing of spv_profile_enable(), and its errors are all returned by the call itself. */
 #define SPV_FILTER_STATIC_BYTES (2u << 20)
 int32_t cls_score_topk_filter_static(const spv_filter_desc* desc, const float* scores,
                                      const void* tokens_in, void* tokens_out, int32_t* kept_idx,
@@ -170,12 +180,16 @@ int32_t cls_score_topk_filter_static(const spv_filter_desc* desc, const float* s
  * Pre-LayerNorm encoder: x = patch_embed(image) + pos;  per block
  *   x += ls1 * (Attn(LN1 x) W_o + b_o);  x += ls2 * MLP(LN2 x);
  * after block `filter_layer` the residual stream is filtered with the CLS scores of that
- * block's attention (Sec. 3.3: pruning after several initial layers, shortening the sequence
- * for all later ones); output = final LayerNorm of the surviving tokens, global tokens first,
- * patches in ascending original position.
+ * block's attention (Sec. 3.3: the pruning comes after a few initial layers and shortens the
+ * sequence for all later ones); output = final LayerNorm of the surviving tokens, global tokens
+ * first, patches in ascending original position.  The filter may be applied at up to
+ * SPV_MAX_FILTERS blocks: every stage ranks the tokens still present by that block's CLS
+ * attention and keeps ceil(keep * present); survivors keep their original grid positions for
+ * the neighbourhood rule of Sec. 3.2.
  * ---------------------------------------------------------------------------------------- */
 enum { SPV_MLP_GELU = 0, SPV_MLP_SWIGLU = 1 };
 enum { SPV_ATTN_DENSE = 0, SPV_ATTN_SPARSE = 1 };
+enum { SPV_MAX_FILTERS = 4 };
 
 typedef struct {
   int32_t layers, dim, heads, mlp_hidden;
@@ -188,6 +202,11 @@ typedef struct {
   int32_t block, radius;
   int32_t filter_layer;   /* 0 = off; f => filter after block f (1-based)                       */
   double keep_ratio;
+  int32_t n_filters;      /* 0: the single stage (filter_layer, keep_ratio) above.  s > 0: stage i
+                             runs after block filter_layers[i] (1-based, strictly increasing) with
+                             keep_ratios[i] in (0, 1]; filter_layer / keep_ratio are ignored      */
+  int32_t filter_layers[SPV_MAX_FILTERS];
+  double keep_ratios[SPV_MAX_FILTERS];
 } spv_vit_config;
 
 /* Per-layer weights: matrices bf16 [out_features, in_features] row-major; vectors fp32. */
@@ -217,10 +236,14 @@ int32_t spv_vit_workspace_size(const spv_vit_config* cfg, int32_t batch, int32_t
                                int32_t grid_w, size_t* bytes);
 
 /* image: fp32 device [batch, 3, grid_h*patch, grid_w*patch], already normalised.
- * out_tokens: bf16 device [batch, n_global + k, dim] (k = grid_h*grid_w when the filter is off).
- * kept_idx: optional int32 device [batch, k] ascending original patch indices.
- * forced_keep: optional int32 device [batch, k] ascending patch indices that replace the
- * ranking (teacher forcing for parity checks).  Asynchronous on `stream`. */
+ * out_tokens: bf16 device [batch, n_global + k, dim], k = tokens left by the last filter stage
+ * (grid_h*grid_w when the filter is off).
+ * kept_idx: optional int32 device [batch, k_1 + ... + k_S]: per image the kept sets of the S
+ * stages one after the other, each as ascending original patch indices (one stage: [batch, k]).
+ * forced_keep: optional int32 device array of the same layout that replaces the ranking of every
+ * stage (teacher forcing for parity checks): each stage's entries strictly ascending, inside the
+ * grid and a subset of the stage before; a violation is found on the device and reported by
+ * spv_check() as SPV_ERR_INVALID_ARG (the output is then undefined).  Asynchronous on `stream`. */
 int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* cfg, const spv_vit_weights* weights,
                     const float* image, int32_t batch, int32_t grid_h, int32_t grid_w,
                     void* out_tokens, int32_t* kept_idx, const int32_t* forced_keep,

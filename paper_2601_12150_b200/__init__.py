@@ -23,7 +23,7 @@ EXPORTS = ["spv_create", "spv_destroy", "spv_status_string", "spv_check", "spv_l
            "spv_filter_keep_count", "spv_filter_workspace_size", "cls_score_topk_filter",
            "cls_score_topk_filter_static",
            "spv_vit_workspace_size", "vit_forward", "spv_gemm_bf16", "spv_layernorm",
-           "spv_profile_enable", "spv_profile_read", "spv_microbench"]
+           "spv_profile_enable", "spv_profile_read", "spv_microbench", "spv_selftest_wait"]
 
 
 class SpvError(RuntimeError):
@@ -51,7 +51,8 @@ class VitConfig(C.Structure):
                 ("mlp_hidden", C.c_int32), ("mlp_kind", C.c_int32), ("patch", C.c_int32),
                 ("n_global", C.c_int32), ("has_layerscale", C.c_int32), ("ln_eps", C.c_float),
                 ("attn_mode", C.c_int32), ("block", C.c_int32), ("radius", C.c_int32),
-                ("filter_layer", C.c_int32), ("keep_ratio", C.c_double)]
+                ("filter_layer", C.c_int32), ("keep_ratio", C.c_double),
+                ("n_filters", C.c_int32), ("filter_layers", C.c_int32 * 4), ("keep_ratios", C.c_double * 4)]
 
 
 LAYER_FIELDS = ["ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_o", "b_o", "ls1", "ln2_g", "ln2_b",
@@ -137,6 +138,7 @@ def lib():
                                     C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
         L.spv_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         L.spv_profile_read.argtypes = [C.c_void_p, C.POINTER(KernelStat)]
+        L.spv_selftest_wait.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         L.spv_microbench.argtypes = [C.c_void_p, C.POINTER(MicrobenchDesc), C.c_void_p, C.c_size_t, C.c_void_p,
                                      C.POINTER(MicrobenchResult)]
         _lib = L
@@ -177,12 +179,34 @@ def cls_score_topk_filter_static(scores, tokens_in, tokens_out, kept_idx, n_glob
     device; calls that may overlap on the GPU must be ordered by the caller (shared scratch).
     scores fp32 [B, h, n_patch]; tokens_in / tokens_out bf16 [B, G+n_patch, dim] / [B, G+k, dim] or
     both None; kept_idx int32 [B, k]."""
+    import torch
     B, H, NP = scores.shape
     dim = 0 if tokens_in is None else tokens_in.shape[-1]
     d = FilterDesc(B, H, NP, n_global, dim, float(keep_ratio), 0, 0)
-    st = lib().cls_score_topk_filter_static(C.byref(d), _ptr(scores), _ptr(tokens_in), _ptr(tokens_out),
-                                            _ptr(kept_idx), _ptr(mean_scores), _ptr(pos_in), _ptr(pos_out),
-                                            _stream(stream))
+    # the library writes k rows / indices per image into the caller's buffers: a buffer of another size, type or
+    # device would be written out of bounds, so check them here (the count fails below if the ratio is invalid)
+    kc = C.c_int32(0)
+    if lib().spv_filter_keep_count(NP, float(keep_ratio), C.byref(kc)) == OK:
+        k = kc.value
+        dev = scores.device
+        assert scores.dtype == torch.float32 and scores.is_contiguous()
+        assert kept_idx.dtype == torch.int32 and kept_idx.is_contiguous() and tuple(kept_idx.shape) == (B, k)
+        assert kept_idx.device == dev
+        if tokens_in is not None:
+            assert tokens_out is not None and tokens_in.dtype == tokens_out.dtype == torch.bfloat16
+            assert tokens_in.is_contiguous() and tokens_out.is_contiguous()
+            assert tuple(tokens_in.shape) == (B, n_global + NP, dim) and tuple(tokens_out.shape) == (B, n_global + k, dim)
+            assert tokens_in.device == dev and tokens_out.device == dev
+        if mean_scores is not None:
+            assert mean_scores.dtype == torch.float32 and mean_scores.is_contiguous() and tuple(mean_scores.shape) == (B, NP)
+        if pos_in is not None:
+            assert pos_out is not None and pos_in.dtype == pos_out.dtype == torch.int32
+            assert tuple(pos_in.shape) == (B, NP) and tuple(pos_out.shape) == (B, k)
+            assert pos_in.is_contiguous() and pos_out.is_contiguous()
+    with torch.cuda.device(scores.device):
+        st = lib().cls_score_topk_filter_static(C.byref(d), _ptr(scores), _ptr(tokens_in), _ptr(tokens_out),
+                                                _ptr(kept_idx), _ptr(mean_scores), _ptr(pos_in), _ptr(pos_out),
+                                                _stream(stream))
     _raise(st, "cls_score_topk_filter_static")
     return tokens_out, kept_idx
 
@@ -341,20 +365,33 @@ class Context:
 
     def vit_forward(self, cfg, dev_weights, image, grid_h, grid_w, forced_keep=None, want_kept=True,
                     out=None, workspace=None, stream=None):
-        """cfg: dict with the spv_vit_config fields.  image fp32 device [B, 3, H*p, W*p].
-        Returns (out_tokens bf16 [B, G+k, dim], kept_idx | None)."""
+        """cfg: dict with the spv_vit_config fields; `filters`: optional list of (layer, keep_ratio) stages
+        in place of filter_layer / keep_ratio.  image fp32 device [B, 3, H*p, W*p].  forced_keep: int32
+        device [B, k_1 + ... + k_S] (the layout of the returned kept array).
+        Returns (out_tokens bf16 [B, G+k, dim], kept int32 [B, k_1 + ... + k_S] | None)."""
         torch = self._torch
+        stages = vit_filter_stages(cfg)
+        multi = bool(cfg.get("filters"))
+        fl = (C.c_int32 * 4)(*([l for l, _ in stages] + [0] * (4 - len(stages)))) if multi else (C.c_int32 * 4)()
+        kr = (C.c_double * 4)(*([r for _, r in stages] + [0.0] * (4 - len(stages)))) if multi else (C.c_double * 4)()
         c = VitConfig(cfg["layers"], cfg["dim"], cfg["heads"], cfg["mlp_hidden"], cfg["mlp_kind"],
                       cfg["patch"], cfg["n_global"], cfg.get("has_layerscale", 0), cfg.get("ln_eps", 1e-6),
                       cfg["attn_mode"], cfg.get("block", 8), cfg.get("radius", 1),
-                      cfg.get("filter_layer", 0), cfg.get("keep_ratio", 1.0))
+                      0 if multi else cfg.get("filter_layer", 0), 1.0 if multi else cfg.get("keep_ratio", 1.0),
+                      len(stages) if multi else 0, fl, kr)
         B = image.shape[0]
         npatch = grid_h * grid_w
-        filt = cfg.get("filter_layer", 0) > 0
-        k = filter_keep_count(npatch, cfg["keep_ratio"]) if filt else npatch
+        counts, cur = [], npatch
+        for _, ratio in stages:
+            cur = filter_keep_count(cur, ratio)
+            counts.append(cur)
+        k = counts[-1] if counts else npatch
         if out is None:
             out = torch.empty((B, cfg["n_global"] + k, cfg["dim"]), dtype=torch.bfloat16, device=image.device)
-        kept = torch.empty((B, k), dtype=torch.int32, device=image.device) if (filt and want_kept) else None
+        kept = torch.empty((B, sum(counts)), dtype=torch.int32, device=image.device) if (counts and want_kept) else None
+        if forced_keep is not None:
+            assert forced_keep.dtype == torch.int32 and forced_keep.is_contiguous()
+            assert tuple(forced_keep.shape) == (B, sum(counts)), "forced_keep: one row of k_1 + ... + k_S per image"
         if workspace is None:
             need = C.c_size_t(0)
             _raise(lib().spv_vit_workspace_size(C.byref(c), B, grid_h, grid_w, C.byref(need)),
@@ -365,6 +402,20 @@ class Context:
                                workspace.numel(), _stream(stream))
         _raise(st, "vit_forward")
         return out, kept
+
+    def selftest_wait(self, limit_ns=200000, stream=None):
+        """Launch the library's one-CTA kernel that waits on a barrier nobody arrives on; the wait gives up
+        after limit_ns and the next check() reports the expired wait."""
+        _raise(lib().spv_selftest_wait(self.handle, int(limit_ns), _stream(stream)), "spv_selftest_wait")
+
+
+def vit_filter_stages(cfg):
+    """[(layer, keep_ratio), ...] of a config dict."""
+    if cfg.get("filters"):
+        return [(int(l), float(r)) for l, r in cfg["filters"]]
+    if cfg.get("filter_layer", 0) > 0:
+        return [(int(cfg["filter_layer"]), float(cfg["keep_ratio"]))]
+    return []
 
 
 class VitWeightsOnDevice:

@@ -69,12 +69,44 @@ __device__ __forceinline__ int lower_bound_blk(const int32_t* pos, int n, int bl
   return lo;
 }
 
+// The caller's positions have to be inside the grid and strictly ascending: by position for row-major
+// callers, by (block, position) for block-major ones (the searches below rely on it).  The first violation
+// is latched in the status word.
+__global__ void attn_check_positions(SpvAttnPlan p, const int32_t* __restrict__ patch_pos, int token_order,
+                                     uint32_t* __restrict__ status) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = blockIdx.y;
+  if (t >= p.n_patch) return;
+  const int32_t* pos = patch_pos + (size_t)b * p.n_patch;
+  const int cur = __ldg(pos + t);
+  bool ok = cur >= 0 && cur < p.grid_h * p.grid_w;
+  if (ok && t > 0) {
+    const int prev = __ldg(pos + t - 1);
+    if (prev < 0 || prev >= p.grid_h * p.grid_w) ok = false;
+    else if (token_order == SPV_TOKENS_ROW_MAJOR) ok = prev < cur;
+    else {
+      const int bp = block_of_pos(prev, p.grid_w, p.block, p.nbx), bc = block_of_pos(cur, p.grid_w, p.block, p.nbx);
+      ok = bp < bc || (bp == bc && prev < cur);
+    }
+  }
+  if (!ok) atomicCAS(status, 0u, SPV_SITE_BAD_PATCH_POS);
+}
+
 // One thread per search segment.  Row-major callers: segment = (block, row inside block): its
 // tokens are one run of the position-sorted input.  Block-major callers: segment = block.
-__global__ void attn_plan_segments(SpvAttnPlan p, const int32_t* __restrict__ patch_pos, int token_order) {
+// `bad` (optional): the word in which attn_check_positions latches a violation; when it is set the plan is
+// built empty (no segment has a token, so no query tile exists and the patch kernel does nothing) instead of
+// being searched for in positions that are not in order.
+__global__ void attn_plan_segments(SpvAttnPlan p, const int32_t* __restrict__ patch_pos, int token_order,
+                                   const uint32_t* __restrict__ bad) {
   const int seg = blockIdx.x * blockDim.x + threadIdx.x;
   const int b = blockIdx.y;
   if (seg >= p.nseg) return;
+  if (bad && *bad != 0u) {
+    p.seg_lo[(size_t)b * p.nseg + seg] = 0;
+    p.seg_cnt[(size_t)b * p.nseg + seg] = 0;
+    return;
+  }
   const int blk = seg / p.segs_per_block, yy = seg % p.segs_per_block;
   const int by = blk / p.nbx, bx = blk % p.nbx;
   const int32_t* pos = patch_pos ? patch_pos + (size_t)b * p.n_patch : nullptr;
@@ -98,7 +130,7 @@ __global__ void attn_plan_segments(SpvAttnPlan p, const int32_t* __restrict__ pa
     }
   }
   p.seg_lo[(size_t)b * p.nseg + seg] = lo;
-  p.seg_cnt[(size_t)b * p.nseg + seg] = cnt;
+  p.seg_cnt[(size_t)b * p.nseg + seg] = max(cnt, 0);
 }
 
 // One CTA per image: exclusive scan of the segment counts, block offsets, then the query tiles.
@@ -178,7 +210,8 @@ __global__ void __launch_bounds__(256) attn_regroup(const __nv_bfloat16* __restr
                                                     int64_t sh, __nv_bfloat16* __restrict__ qo,
                                                     __nv_bfloat16* __restrict__ ko, __nv_bfloat16* __restrict__ vo,
                                                     const int32_t* __restrict__ bm_src, int batch, int n_global,
-                                                    int n_patch, int heads) {
+                                                    int n_patch, int heads, const uint32_t* __restrict__ bad) {
+  if (*bad != 0u) return;        // the plan is empty (positions out of order): bm_src holds nothing
   const int n_tok = n_global + n_patch;
   const int64_t total = (int64_t)batch * n_tok * heads;
   const int sub = threadIdx.x & 7;
@@ -754,7 +787,7 @@ __global__ void __launch_bounds__(256) attn_global_combine(const float* __restri
                                                            int n_tok, int n_global, int heads,
                                                            __nv_bfloat16* __restrict__ o, int64_t o_sb,
                                                            int64_t o_st, int64_t o_sh, float* __restrict__ scores,
-                                                           const int32_t* __restrict__ score_idx) {
+                                                           const int32_t* __restrict__ score_idx, int score_stride) {
   __shared__ float s_m, s_l;
   __shared__ float s_red[16];
   const int h = blockIdx.x, bg = blockIdx.y;
@@ -796,7 +829,7 @@ __global__ void __launch_bounds__(256) attn_global_combine(const float* __restri
   if (scores && g == 0) {
     const float* lg = logits + ((size_t)bg * heads + h) * n_tok;
     const int n_patch = n_tok - n_global;
-    float* sc = scores + ((size_t)b * heads + h) * n_patch;
+    float* sc = scores + ((size_t)b * heads + h) * score_stride;
     for (int t = threadIdx.x; t < n_patch; t += 256) {
       const int dst = score_idx ? __ldg(score_idx + (size_t)b * n_patch + t) : t;
       sc[dst] = __expf(lg[n_global + t] - M) * inv;
@@ -846,7 +879,7 @@ size_t spv_attn_plan_bytes(int32_t batch, int32_t grid_h, int32_t grid_w, int32_
 int32_t spv_attn_plan_build(spv_ctx* ctx, int32_t batch, int32_t grid_h, int32_t grid_w, int32_t block,
                             int32_t radius, int32_t n_global, int32_t n_patch, const int32_t* patch_pos,
                             int32_t token_order, void* ws, size_t ws_bytes, cudaStream_t stream,
-                            SpvAttnPlan* plan) {
+                            SpvAttnPlan* plan, bool check_positions) {
   SpvAttnPlan p{};
   p.batch = batch; p.grid_h = grid_h; p.grid_w = grid_w; p.block = block; p.n_global = n_global;
   p.n_patch = n_patch;
@@ -866,11 +899,18 @@ int32_t spv_attn_plan_build(spv_ctx* ctx, int32_t batch, int32_t grid_h, int32_t
   p.tiles = (int4*)take((size_t)batch * p.tiles_per_image * sizeof(int4));
   const dim3 sgrid((p.nseg + 255) / 256, batch);
   SpvProfScope prof(ctx, SPV_K_ATTN_PLAN, stream);
-  attn_plan_segments<<<sgrid, 256, 0, stream>>>(p, patch_pos, token_order);
+  int launches = 3;
+  if (check_positions && patch_pos) {
+    attn_check_positions<<<dim3((n_patch + 255) / 256, batch), 256, 0, stream>>>(p, patch_pos, token_order,
+                                                                              ctx->d_status + 1);
+    ++launches;
+  }
+  attn_plan_segments<<<sgrid, 256, 0, stream>>>(p, patch_pos, token_order,
+                                                (check_positions && patch_pos) ? ctx->d_status + 1 : nullptr);
   attn_plan_scan<<<batch, 1024, 0, stream>>>(p);
   attn_plan_fill<<<sgrid, 256, 0, stream>>>(p);
   *plan = p;
-  return spv_launch_ok(ctx, 3);
+  return spv_launch_ok(ctx, launches);
 }
 
 int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, cudaStream_t stream) {
@@ -913,7 +953,8 @@ size_t spv_attn_global_bytes(int32_t batch, int32_t n_global, int32_t heads, int
 }
 
 int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, float* scores,
-                             const int32_t* score_idx, void* ws, size_t ws_bytes, cudaStream_t stream) {
+                             const int32_t* score_idx, int32_t score_stride, void* ws, size_t ws_bytes,
+                             cudaStream_t stream) {
   const int n_tok = plan->n_global + plan->n_patch, G = plan->n_global, B = plan->batch;
   if (ws_bytes < spv_attn_global_bytes(B, G, io->heads, n_tok)) return SPV_ERR_WORKSPACE;
   const size_t rows = (size_t)B * G * io->heads;
@@ -936,7 +977,7 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
       n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks, chunk_len);
   attn_global_combine<<<dim3(io->heads, B * G), 256, 0, stream>>>(logits, part_ml, part_o, chunks, n_tok, G,
                                                                  io->heads, (__nv_bfloat16*)io->o, io->o_sb,
-                                                                 io->o_st, io->o_sh, scores, score_idx);
+                                                                 io->o_st, io->o_sh, scores, score_idx, score_stride);
   return spv_launch_ok(ctx, 2);
 }
 
@@ -988,7 +1029,7 @@ extern "C" int32_t spatial_block_attention(spv_ctx* ctx, const spv_attn_desc* d,
   const size_t plan_b = spv_attn_plan_bytes(d->batch, d->grid_h, d->grid_w, d->block, d->n_patch, d->token_order);
   SpvAttnPlan plan;
   st = spv_attn_plan_build(ctx, d->batch, d->grid_h, d->grid_w, d->block, d->radius, d->n_global, d->n_patch,
-                           d->patch_pos, d->token_order, w, plan_b, stream, &plan);
+                           d->patch_pos, d->token_order, w, plan_b, stream, &plan, true);
   if (st != SPV_OK) return st;
   w += plan_b;
   const int n_tok = d->n_global + d->n_patch;
@@ -1013,7 +1054,7 @@ extern "C" int32_t spatial_block_attention(spv_ctx* ctx, const spv_attn_desc* d,
     attn_regroup<<<(unsigned)blocks, 256, 0, stream>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                                       (const __nv_bfloat16*)v, d->stride_b, d->stride_tok,
                                                       d->stride_head, qb, kb, vb, plan.bm_src, d->batch,
-                                                      d->n_global, d->n_patch, d->heads);
+                                                      d->n_global, d->n_patch, d->heads, ctx->d_status + 1);
     if ((st = spv_launch_ok(ctx)) != SPV_OK) return st;
     io.q = qb; io.k = kb; io.v = vb;
     io.st = (int64_t)d->heads * HD; io.sh = HD; io.sb = (int64_t)n_tok * d->heads * HD;
@@ -1023,6 +1064,6 @@ extern "C" int32_t spatial_block_attention(spv_ctx* ctx, const spv_attn_desc* d,
     io.o_tok = nullptr;
   }
   if ((st = spv_attn_run_patches(ctx, &plan, &io, stream)) != SPV_OK) return st;
-  return spv_attn_run_globals(ctx, &plan, &gio, cls_scores, nullptr, w,
+  return spv_attn_run_globals(ctx, &plan, &gio, cls_scores, nullptr, d->n_patch, w,
                               spv_attn_global_bytes(d->batch, d->n_global, d->heads, n_tok), stream);
 }

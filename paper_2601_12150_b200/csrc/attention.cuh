@@ -23,11 +23,12 @@ struct SpvAttnPlan {
 size_t spv_attn_plan_bytes(int32_t batch, int32_t grid_h, int32_t grid_w, int32_t block, int32_t n_patch,
                            int32_t token_order);
 
-// Build the plan on `stream` (three small kernels).  patch_pos as in spv_attn_desc.
+// Build the plan on `stream` (three small kernels).  patch_pos as in spv_attn_desc; check_positions adds a
+// kernel that verifies a caller's patch_pos (range and order) and latches a violation in the status word.
 int32_t spv_attn_plan_build(spv_ctx* ctx, int32_t batch, int32_t grid_h, int32_t grid_w, int32_t block,
                             int32_t radius, int32_t n_global, int32_t n_patch, const int32_t* patch_pos,
                             int32_t token_order, void* ws, size_t ws_bytes, cudaStream_t stream,
-                            SpvAttnPlan* plan);
+                            SpvAttnPlan* plan, bool check_positions = false);
 
 struct SpvAttnIO {
   const void *q, *k, *v;            // bf16, tokens in BLOCK-MAJOR order (globals first)
@@ -43,7 +44,10 @@ struct SpvAttnIO {
 int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, cudaStream_t stream);
 
 // Global-query rows (dense rows, memory-bound) and optional CLS->patch scores.
-// scores: fp32 [B][heads][n_patch] indexed by score_idx[b][t] (NULL = t) for block-major ordinal t.
+// scores: fp32 [B][heads][score_stride], the weight of block-major ordinal t written at score_idx[b][t]
+// (NULL = t); score_stride >= the largest index + 1 (the patch count, or the grid size when the indices
+// are original positions).
 size_t spv_attn_global_bytes(int32_t batch, int32_t n_global, int32_t heads, int32_t n_tok);
 int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, float* scores,
-                             const int32_t* score_idx, void* ws, size_t ws_bytes, cudaStream_t stream);
+                             const int32_t* score_idx, int32_t score_stride, void* ws, size_t ws_bytes,
+                             cudaStream_t stream);

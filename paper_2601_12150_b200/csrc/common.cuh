@@ -20,7 +20,8 @@ typedef CUresult (*spv_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuin
 struct spv_ctx {
   int32_t device;
   int32_t sm_count;
-  uint32_t* d_status;            // device status word: 0 = ok, else first failing site code
+  uint32_t* d_status;            // device status words: [0] 0 = ok, else site code of the first expired wait;
+                                 // [1] 0 = ok, else code of the first bad caller index array
   spv_encode_tiled_fn encode_tiled;
   int64_t launches;
   uint32_t last_site;            // site code read by the last failing spv_check
@@ -42,6 +43,12 @@ struct SpvProfScope {
       : ctx(c), stream(s), token(c->prof_on ? spv_prof_begin(c, cls, s) : -1), work(w) {}
   ~SpvProfScope() { if (token >= 0) spv_prof_end(ctx, token, stream, work); }
 };
+
+// Second device status word (d_status[1]; the bounded waits look at d_status[0] only): an index array given
+// by the caller broke its documented range or order, found by the kernel that reads it.  spv_check() reports
+// these as SPV_ERR_INVALID_ARG.
+#define SPV_SITE_BAD_KEPT_INDEX 0xB001u   // forced_keep of vit_forward
+#define SPV_SITE_BAD_PATCH_POS 0xB002u    // patch_pos of spatial_block_attention
 
 #define SPV_CUDA_OK(expr)                         \
   do {                                            \

@@ -118,14 +118,39 @@ extern "C" const char* spv_status_string(int32_t s) {
 extern "C" int32_t spv_check(spv_ctx* ctx, void* stream) {
   if (!ctx) return SPV_ERR_INVALID_ARG;
   SPV_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
-  uint32_t st = 0;
-  SPV_CUDA_OK(cudaMemcpy(&st, ctx->d_status, sizeof(st), cudaMemcpyDeviceToHost));
-  if (st != 0) {
-    ctx->last_site = st;
+  uint32_t st[2] = {0, 0};
+  SPV_CUDA_OK(cudaMemcpy(st, ctx->d_status, sizeof(st), cudaMemcpyDeviceToHost));
+  if (st[0] != 0 || st[1] != 0) {
+    ctx->last_site = st[0] != 0 ? st[0] : st[1];
     cudaMemset(ctx->d_status, 0, sizeof(st));
-    return SPV_ERR_TIMEOUT;
+    return st[0] != 0 ? SPV_ERR_TIMEOUT : SPV_ERR_INVALID_ARG;
   }
   return SPV_OK;
+}
+
+// One thread waits on a barrier that gets no arrival, for at most limit_ns: the same parked try_wait and the
+// same latch as the kernels' bounded waits, with the limit as an argument.
+__global__ void selftest_wait_kernel(uint32_t limit_ns, uint32_t* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    spv::mbar_init(&bar, 1);
+    spv::mbar_fence_init();
+    uint32_t t0, t;
+    asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t0));
+    bool done = false;
+    do {
+      done = spv::mbar_try_wait_parked(&bar, 0, 1000u);
+      asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t));
+    } while (!done && t - t0 <= limit_ns);
+    if (!done) atomicCAS(status, 0u, 0x5E1Fu);
+  }
+}
+
+extern "C" int32_t spv_selftest_wait(spv_ctx* ctx, uint32_t limit_ns, void* stream) {
+  if (!ctx) return SPV_ERR_INVALID_ARG;
+  if (limit_ns > 1000000u) limit_ns = 1000000u;
+  selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_ns, ctx->d_status);
+  return spv_launch_ok(ctx);
 }
 
 extern "C" uint32_t spv_last_wait_site(const spv_ctx* ctx) { return ctx ? ctx->last_site : 0u; }

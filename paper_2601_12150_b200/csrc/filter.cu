@@ -7,7 +7,7 @@
 //   filter_select     one CTA per image: 4-pass radix select of the k-th largest key, then an
 //                     ordered two-counter scan that emits the kept indices in ascending order;
 //   filter_gather     128-bit row copy of the global tokens and the kept rows.
-#include "common.cuh"
+#include "filter.cuh"
 
 namespace {
 
@@ -226,15 +226,22 @@ extern "C" int32_t cls_score_topk_filter(spv_ctx* ctx, const spv_filter_desc* d,
   int32_t k;
   int32_t st = validate(d, &k);
   if (st != SPV_OK) return st;
+  return spv_filter_run_k(ctx, d, k, scores, tokens_in, tokens_out, kept_idx, mean_scores, pos_in, pos_out, workspace,
+                          workspace_bytes, (cudaStream_t)stream_);
+}
+
+int32_t spv_filter_run_k(spv_ctx* ctx, const spv_filter_desc* d, int32_t k, const float* scores,
+                         const void* tokens_in, void* tokens_out, int32_t* kept_idx, float* mean_scores,
+                         const int32_t* pos_in, int32_t* pos_out, void* workspace, size_t workspace_bytes,
+                         cudaStream_t stream) {
+  if (!ctx || !d || k < 1 || k > d->n_patch) return SPV_ERR_INVALID_ARG;
   if (!scores || !kept_idx) return SPV_ERR_INVALID_ARG;
   if ((tokens_in == nullptr) != (tokens_out == nullptr)) return SPV_ERR_INVALID_ARG;
   if (tokens_in && d->dim == 0) return SPV_ERR_INVALID_ARG;
   if (((uintptr_t)scores & 15u) || ((uintptr_t)tokens_in & 15u) || ((uintptr_t)tokens_out & 15u))
     return SPV_ERR_ALIGNMENT;
-  size_t need;
-  spv_filter_workspace_size(d, &need);
+  const size_t need = spv_align_up((size_t)d->batch * spv_align_up((size_t)d->n_patch, 4) * sizeof(float), 256) * 2;
   if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255u)) return SPV_ERR_WORKSPACE;
-  cudaStream_t stream = (cudaStream_t)stream_;
   const int npad = (int)spv_align_up((size_t)d->n_patch, 4);
   float* mean_ws = (float*)workspace;
   uint32_t* key_ws =

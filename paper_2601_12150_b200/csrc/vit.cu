@@ -10,6 +10,7 @@
 // The residual stream stays fp32 (LayerNorm reads it, the GEMM epilogues add into it); every
 // GEMM operand is bf16.
 #include "attention.cuh"
+#include "filter.cuh"
 
 namespace {
 
@@ -108,23 +109,31 @@ __global__ void vit_pad_weight(const __nv_bfloat16* __restrict__ w, int rows, in
   w_pad[i] = c < kp ? w[(int64_t)r * kp + c] : __float2bfloat16(0.f);
 }
 
-// mark[b, pos] = 1 for every kept original position (mark zeroed beforehand)
-__global__ void vit_mark_kept(const int32_t* __restrict__ kept, int k, int np, float* __restrict__ mark) {
+// mark[b, pos] = 1 for every kept original position (mark zeroed beforehand).  kept: [batch] rows of k
+// entries, `stride` apart.  The entries have to be inside the grid, strictly ascending and, for a later
+// stage, marked by the stage before (prev_mark); the first violation is latched in the status word.
+__global__ void vit_mark_kept(const int32_t* __restrict__ kept, int64_t stride, int k, int np,
+                              float* __restrict__ mark, const float* __restrict__ prev_mark,
+                              uint32_t* __restrict__ status) {
   const int b = blockIdx.y;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= k) return;
-  const int pos = __ldg(kept + (size_t)b * k + i);
-  if (pos >= 0 && pos < np) mark[(size_t)b * np + pos] = 1.0f;
+  const int pos = __ldg(kept + (size_t)b * stride + i);
+  bool ok = pos >= 0 && pos < np;
+  if (ok && i > 0) ok = __ldg(kept + (size_t)b * stride + i - 1) < pos;
+  if (ok && prev_mark) ok = prev_mark[(size_t)b * np + pos] != 0.0f;
+  if (ok) mark[(size_t)b * np + pos] = 1.0f;
+  else atomicCAS(status, 0u, SPV_SITE_BAD_KEPT_INDEX);
 }
 
-// mask_bm[b, t] = mark[b, bm_pos[b, t]]: the kept set as a one-head score row over the internal
-// token order; ranking it keeps exactly the marked tokens, in internal order.
-__global__ void vit_mask_to_order(const float* __restrict__ mark, const int32_t* __restrict__ bm_pos, int np,
-                                  float* __restrict__ mask_bm) {
+// mask_bm[b, t] = mark[b, cur_pos[b, t]] for the n_cur tokens present: the kept set as a one-head score
+// row over the internal token order; ranking it keeps exactly the marked tokens, in internal order.
+__global__ void vit_mask_to_order(const float* __restrict__ mark, const int32_t* __restrict__ cur_pos, int n_cur,
+                                  int np_grid, float* __restrict__ mask_bm) {
   const int b = blockIdx.y;
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= np) return;
-  mask_bm[(size_t)b * np + t] = mark[(size_t)b * np + __ldg(bm_pos + (size_t)b * np + t)];
+  if (t >= n_cur) return;
+  mask_bm[(size_t)b * n_cur + t] = mark[(size_t)b * np_grid + __ldg(cur_pos + (size_t)b * n_cur + t)];
 }
 
 // Destination row of every internal row for the final LayerNorm.  Unfiltered: G + position.
@@ -182,9 +191,11 @@ __global__ void __launch_bounds__(1024) vit_out_rows_kept(const float* __restric
 // workspace layout
 // ------------------------------------------------------------------------------------------
 struct VitLayout {
-  int32_t np0, n0, k, n1, kp, kpad, nbx, nby;
-  size_t x0, x1, h, qkv, o, h1, h3, im2col, w_pe_pad, pos_bm, scores, mask, mark, rank, bm_pos, bm_of_pos, pos2,
-      kept_bm, kept_rm, out_row, plan, plan_bytes, glob, glob_bytes, filt, filt_bytes, total;
+  int32_t np0, n0, k, k1, n1, kp, kpad, nbx, nby;
+  // filter stages: block after which each runs, tokens it keeps, entries per image over all stages
+  int32_t n_stage, st_layer[SPV_MAX_FILTERS], st_k[SPV_MAX_FILTERS], k_total;
+  size_t x0, x1, h, qkv, o, h1, h3, im2col, w_pe_pad, pos_bm, scores, mask, mark, mark2, rank, bm_pos, bm_of_pos, pos2,
+      pos3, kept_bm, kept_rm, out_row, plan, plan_bytes, glob, glob_bytes, filt, filt_bytes, total;
 };
 
 int32_t vit_layout(const spv_vit_config* c, int32_t batch, int32_t gh, int32_t gw, VitLayout* L) {
@@ -196,17 +207,36 @@ int32_t vit_layout(const spv_vit_config* c, int32_t batch, int32_t gh, int32_t g
   if (c->mlp_kind != SPV_MLP_GELU && c->mlp_kind != SPV_MLP_SWIGLU) return SPV_ERR_INVALID_ARG;
   if (c->attn_mode != SPV_ATTN_DENSE && c->attn_mode != SPV_ATTN_SPARSE) return SPV_ERR_INVALID_ARG;
   if (c->block < 1 || c->radius < 0) return SPV_ERR_INVALID_ARG;
-  if (c->filter_layer < 0 || c->filter_layer > c->layers) return SPV_ERR_INVALID_ARG;
   if ((int64_t)gh * gw > (1 << 24)) return SPV_ERR_UNSUPPORTED;
   const int32_t G = c->n_global, D = c->dim, HID = c->mlp_hidden;
   L->np0 = gh * gw;
   L->n0 = G + L->np0;
-  L->k = L->np0;
-  if (c->filter_layer > 0) {
-    int32_t st = spv_filter_keep_count(L->np0, c->keep_ratio, &L->k);
-    if (st != SPV_OK) return st;
+  // the filter stages
+  double st_keep[SPV_MAX_FILTERS];
+  L->n_stage = 0;
+  if (c->n_filters < 0 || c->n_filters > SPV_MAX_FILTERS) return SPV_ERR_INVALID_ARG;
+  if (c->n_filters == 0) {
+    if (c->filter_layer < 0 || c->filter_layer > c->layers) return SPV_ERR_INVALID_ARG;
+    if (c->filter_layer > 0) { L->n_stage = 1; L->st_layer[0] = c->filter_layer; st_keep[0] = c->keep_ratio; }
+  } else {
+    L->n_stage = c->n_filters;
+    for (int s = 0; s < L->n_stage; ++s) {
+      L->st_layer[s] = c->filter_layers[s];
+      st_keep[s] = c->keep_ratios[s];
+      if (L->st_layer[s] < 1 || L->st_layer[s] > c->layers) return SPV_ERR_INVALID_ARG;
+      if (s > 0 && L->st_layer[s] <= L->st_layer[s - 1]) return SPV_ERR_INVALID_ARG;
+    }
   }
-  L->n1 = G + L->k;
+  L->k = L->np0;
+  L->k_total = 0;
+  for (int s = 0; s < L->n_stage; ++s) {
+    int32_t st = spv_filter_keep_count(L->k, st_keep[s], &L->st_k[s]);
+    if (st != SPV_OK) return st;
+    L->k = L->st_k[s];
+    L->k_total += L->k;
+  }
+  L->k1 = L->n_stage > 0 ? L->st_k[0] : L->np0;      // the longest sequence after a filter
+  L->n1 = G + L->k1;
   L->kp = 3 * c->patch * c->patch;
   L->kpad = (int32_t)spv_align_up((size_t)L->kp, 8);
   L->nby = (gh + c->block - 1) / c->block;
@@ -215,7 +245,7 @@ int32_t vit_layout(const spv_vit_config* c, int32_t batch, int32_t gh, int32_t g
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t r = off; off += spv_align_up(bytes, 256); return r; };
   L->x0 = take(rows * D * 4);
-  L->x1 = take(c->filter_layer > 0 ? (size_t)batch * L->n1 * D * 4 : 0);
+  L->x1 = take(L->n_stage > 0 ? (size_t)batch * L->n1 * D * 4 : 0);
   L->h = take(rows * D * 2);
   L->qkv = take(rows * 3 * D * 2);
   L->o = take(rows * D * 2);
@@ -229,12 +259,14 @@ int32_t vit_layout(const spv_vit_config* c, int32_t batch, int32_t gh, int32_t g
   L->scores = take((size_t)batch * c->heads * L->np0 * 4);
   L->mask = take((size_t)batch * L->np0 * 4);
   L->mark = take((size_t)batch * L->np0 * 4);
+  L->mark2 = take(L->n_stage > 1 ? (size_t)batch * L->np0 * 4 : 0);
   L->rank = take((size_t)batch * L->np0 * 4);
   L->bm_pos = take((size_t)batch * L->np0 * 4);
   L->bm_of_pos = take((size_t)L->np0 * 4);
-  L->pos2 = take((size_t)batch * L->k * 4);
-  L->kept_bm = take((size_t)batch * L->k * 4);
-  L->kept_rm = take((size_t)batch * L->k * 4);
+  L->pos2 = take((size_t)batch * L->k1 * 4);
+  L->pos3 = take(L->n_stage > 1 ? (size_t)batch * L->k1 * 4 : 0);
+  L->kept_bm = take((size_t)batch * L->k1 * 4);
+  L->kept_rm = take((size_t)batch * L->k1 * 4);
   L->out_row = take(rows * 4);
   L->plan_bytes = spv_attn_plan_bytes(batch, gh, gw, c->block, L->np0, SPV_TOKENS_BLOCK_MAJOR);
   L->plan = take(L->plan_bytes);
@@ -242,7 +274,7 @@ int32_t vit_layout(const spv_vit_config* c, int32_t batch, int32_t gh, int32_t g
   L->glob = take(L->glob_bytes);
   spv_filter_desc fd{};
   fd.batch = batch; fd.heads = c->heads; fd.n_patch = L->np0; fd.n_global = G; fd.dim = 2 * D;
-  fd.keep_ratio = c->filter_layer > 0 ? c->keep_ratio : 1.0;
+  fd.keep_ratio = 1.0;
   size_t fb = 0;
   int32_t st = spv_filter_workspace_size(&fd, &fb);
   if (st != SPV_OK) return st;
@@ -274,7 +306,7 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
   int32_t st = vit_layout(c, batch, gh, gw, &L);
   if (st != SPV_OK) return st;
   if (!workspace || workspace_bytes < L.total || ((uintptr_t)workspace & 255u)) return SPV_ERR_WORKSPACE;
-  if (forced_keep && c->filter_layer == 0) return SPV_ERR_INVALID_ARG;
+  if (forced_keep && L.n_stage == 0) return SPV_ERR_INVALID_ARG;
   if (!w->w_pe || !w->cls || !w->pos || !w->lnf_g || !w->lnf_b) return SPV_ERR_INVALID_ARG;
   if (((uintptr_t)image & 15u) || ((uintptr_t)out_tokens & 15u)) return SPV_ERR_ALIGNMENT;
   cudaStream_t stream = (cudaStream_t)stream_;
@@ -294,10 +326,12 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
   float* scores = (float*)(ws + L.scores);
   float* mask = (float*)(ws + L.mask);
   float* mark = (float*)(ws + L.mark);
+  float* mark2 = (float*)(ws + L.mark2);
   int32_t* rank = (int32_t*)(ws + L.rank);
   int32_t* bm_pos = (int32_t*)(ws + L.bm_pos);
   int32_t* bm_of_pos = (int32_t*)(ws + L.bm_of_pos);
   int32_t* pos2 = (int32_t*)(ws + L.pos2);
+  int32_t* pos3 = (int32_t*)(ws + L.pos3);
   int32_t* kept_bm = (int32_t*)(ws + L.kept_bm);
   int32_t* kept_rm = (int32_t*)(ws + L.kept_rm);
   int32_t* out_row = (int32_t*)(ws + L.out_row);
@@ -345,6 +379,9 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
   int32_t np = np0;            // patch tokens currently present
   int64_t n = L.n0;            // tokens per image
   const int32_t* cur_pos = bm_pos;
+  int stage = 0;               // next filter stage
+  int32_t k_before = 0;        // entries of the earlier stages in kept_idx / forced_keep
+  const float* last_mark = nullptr;
   for (int l = 1; l <= c->layers; ++l) {
     const spv_layer_weights* lw = &w->layer[l - 1];
     if (!lw->ln1_g || !lw->ln1_b || !lw->w_qkv || !lw->w_o || !lw->ln2_g || !lw->ln2_b || !lw->w_fc1 || !lw->w_fc2)
@@ -369,9 +406,12 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
       if ((st = spv_attn_run_patches(ctx, &plan, &io, stream)) != SPV_OK) return st;
       // CLS->patch scores land at the tokens' ORIGINAL positions, so that the ranking breaks
       // ties by the lower original index
-      const bool want_scores = (l == c->filter_layer) && !forced_keep;
+      const bool want_scores = stage < L.n_stage && l == L.st_layer[stage] && !forced_keep;
+      // a later stage ranks over the whole grid: positions that are gone hold NaN, which ranks last
+      if (want_scores && stage > 0)
+        SPV_CUDA_OK(cudaMemsetAsync(scores, 0xFF, (size_t)batch * H * np0 * 4, stream));
       if ((st = spv_attn_run_globals(ctx, &plan, &io, want_scores ? scores : nullptr, want_scores ? cur_pos : nullptr,
-                                     ws + L.glob, L.glob_bytes, stream)) != SPV_OK)
+                                     np0, ws + L.glob, L.glob_bytes, stream)) != SPV_OK)
         return st;
     }
     {
@@ -402,41 +442,55 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
       if ((st = spv_gemm_bf16(ctx, &g, mlp_act, lw->w_fc2, x, stream)) != SPV_OK) return st;
     }
 
-    // ---- Sec. 3.3: after block `filter_layer` the lowest-scored patches leave the sequence (a8-a10)
-    if (l == c->filter_layer) {
-      const int32_t k = L.k;
-      const int32_t* kept_positions = forced_keep;
-      if (!forced_keep) {
+    // ---- Sec. 3.3: after a stage's block the lowest-scored patches leave the sequence (a8-a10)
+    if (stage < L.n_stage && l == L.st_layer[stage]) {
+      const int32_t k = L.st_k[stage];
+      const int32_t* kept_positions;
+      int64_t kept_stride;
+      if (forced_keep) {
+        kept_positions = forced_keep + k_before;
+        kept_stride = L.k_total;
+      } else {
         // rank on the head-averaged scores in original-position order -> ascending original indices
         spv_filter_desc fd{};
-        fd.batch = batch; fd.heads = H; fd.n_patch = np0; fd.n_global = G; fd.dim = 0; fd.keep_ratio = c->keep_ratio;
-        if ((st = cls_score_topk_filter(ctx, &fd, scores, nullptr, nullptr, kept_rm, nullptr, nullptr, nullptr,
-                                        ws + L.filt, L.filt_bytes, stream)) != SPV_OK)
+        fd.batch = batch; fd.heads = H; fd.n_patch = np0; fd.n_global = G; fd.dim = 0; fd.keep_ratio = 1.0;
+        if ((st = spv_filter_run_k(ctx, &fd, k, scores, nullptr, nullptr, kept_rm, nullptr, nullptr, nullptr,
+                                   ws + L.filt, L.filt_bytes, stream)) != SPV_OK)
           return st;
         kept_positions = kept_rm;
+        kept_stride = k;
       }
       // the kept set as a one-head score row over the internal order; ranking it compacts the
       // residual stream (fp32 rows copied as 2*D 16-bit elements) and the positions, order kept
+      float* mk = (stage & 1) ? mark2 : mark;
       {
         SpvProfScope prof(ctx, SPV_K_MISC, stream);
-        SPV_CUDA_OK(cudaMemsetAsync(mark, 0, (size_t)batch * np0 * 4, stream));
-        vit_mark_kept<<<dim3(cdiv(k, 256), batch), 256, 0, stream>>>(kept_positions, k, np0, mark);
-        vit_mask_to_order<<<dim3(cdiv(np0, 256), batch), 256, 0, stream>>>(mark, bm_pos, np0, mask);
+        SPV_CUDA_OK(cudaMemsetAsync(mk, 0, (size_t)batch * np0 * 4, stream));
+        vit_mark_kept<<<dim3(cdiv(k, 256), batch), 256, 0, stream>>>(kept_positions, kept_stride, k, np0, mk, last_mark,
+                                                                     ctx->d_status + 1);
+        vit_mask_to_order<<<dim3(cdiv(np, 256), batch), 256, 0, stream>>>(mk, cur_pos, np, np0, mask);
       }
       if ((st = spv_launch_ok(ctx, 2)) != SPV_OK) return st;
+      float* x_next = (x == (float*)(ws + L.x0)) ? x_alt : (float*)(ws + L.x0);
+      int32_t* pos_next = (cur_pos == pos2) ? pos3 : pos2;
       spv_filter_desc fd{};
-      fd.batch = batch; fd.heads = 1; fd.n_patch = np0; fd.n_global = G; fd.dim = 2 * D; fd.keep_ratio = c->keep_ratio;
-      fd.in_stride_b = (int64_t)L.n0 * 2 * D; fd.out_stride_b = (int64_t)L.n1 * 2 * D;
-      if ((st = cls_score_topk_filter(ctx, &fd, mask, x, x_alt, kept_bm, nullptr, bm_pos, pos2, ws + L.filt,
-                                      L.filt_bytes, stream)) != SPV_OK)
+      fd.batch = batch; fd.heads = 1; fd.n_patch = np; fd.n_global = G; fd.dim = 2 * D; fd.keep_ratio = 1.0;
+      fd.in_stride_b = n * 2 * D; fd.out_stride_b = (int64_t)(G + k) * 2 * D;
+      if ((st = spv_filter_run_k(ctx, &fd, k, mask, x, x_next, kept_bm, nullptr, cur_pos, pos_next, ws + L.filt,
+                                 L.filt_bytes, stream)) != SPV_OK)
         return st;
       if (kept_idx)
-        SPV_CUDA_OK(cudaMemcpyAsync(kept_idx, kept_positions, (size_t)batch * k * 4, cudaMemcpyDeviceToDevice, stream));
-      x = x_alt;
+        SPV_CUDA_OK(cudaMemcpy2DAsync(kept_idx + k_before, (size_t)L.k_total * 4, kept_positions,
+                                      (size_t)kept_stride * 4, (size_t)k * 4, (size_t)batch, cudaMemcpyDeviceToDevice,
+                                      stream));
+      x = x_next;
       np = k;
-      n = L.n1;
-      cur_pos = pos2;
-      if ((st = spv_attn_plan_build(ctx, batch, gh, gw, c->block, radius, G, np, pos2, SPV_TOKENS_BLOCK_MAJOR,
+      n = G + k;
+      cur_pos = pos_next;
+      last_mark = mk;
+      k_before += k;
+      ++stage;
+      if ((st = spv_attn_plan_build(ctx, batch, gh, gw, c->block, radius, G, np, cur_pos, SPV_TOKENS_BLOCK_MAJOR,
                                     ws + L.plan, L.plan_bytes, stream, &plan)) != SPV_OK)
         return st;
     }
@@ -445,8 +499,8 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
   // ---- final LayerNorm, rows scattered back to ascending original position (a12)
   {
     SpvProfScope prof(ctx, SPV_K_MISC, stream);
-    if (c->filter_layer > 0) {
-      vit_out_rows_kept<<<batch, 1024, 0, stream>>>(mark, np0, pos2, L.k, G, rank, out_row);
+    if (L.n_stage > 0) {
+      vit_out_rows_kept<<<batch, 1024, 0, stream>>>(last_mark, np0, cur_pos, L.k, G, rank, out_row);
     } else {
       vit_out_rows_full<<<dim3(cdiv(L.n0, 256), batch), 256, 0, stream>>>(bm_pos, G, np0, out_row);
     }

@@ -21,9 +21,12 @@ def ctx():
 
 
 def _check(got, ref, max_abs=2e-2, rel_l2=5e-3):
+    """max |err| <= 2e-2 and relative L2 <= 5e-3; above |ref| = 2 the element bound is 1e-2 |ref| (half an ulp
+    of the bf16 output is up to 2^-8 |x|, which alone passes 2e-2 from |x| = 5.1 on)."""
     err = got.astype(np.float64) - ref.astype(np.float64)
     assert np.isfinite(got).all()
-    assert np.abs(err).max() <= max_abs, np.abs(err).max()
+    bound = np.maximum(max_abs, 0.5 * max_abs * np.abs(ref.astype(np.float64)))
+    assert (np.abs(err) <= bound).all(), float((np.abs(err) / bound).max())
     rel = np.linalg.norm(err) / np.linalg.norm(ref)
     assert rel <= rel_l2, rel
 
@@ -160,7 +163,7 @@ def test_large_scores_and_argument_errors(ctx):
     q, k, v = synth.attention_qkv(21, 1, 1 + 256, 2, 64, std=2.5)
     want, _ = oracle.attention(q, k, v, 16, 16, 8, 1)
     got, _ = _run(ctx, q, k, v, 16, 16, 8, 1)
-    _check(got, want, max_abs=4e-2)
+    _check(got, want)
     dq = torch.zeros((1, 17, 2, 32), dtype=torch.bfloat16, device=ctx.device)
     with pytest.raises(spv.SpvError) as e:
         ctx.spatial_block_attention(dq, dq, dq, 4, 4, 2, 1)

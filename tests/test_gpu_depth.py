@@ -1,0 +1,86 @@
+"""vit_forward against the oracle at the full depth of the benchmark configurations: bf16 operands and an
+fp32 residual stream over 24 and 40 blocks against the oracle's fp32/fp64 arithmetic, tolerance unchanged
+(max |err| <= 2e-2, relative L2 <= 5e-3), free-running then teacher-forced as in test_gpu_vit.
+
+ViT-L/16 at 1024x1024 (24 blocks, 64x64 grid; dense, sparse, sparse + filter keep 0.6 after block 4) runs
+by default.  One image of the 2048x2048 benchmark workload and the ViT-g/14-style forward (40 blocks,
+146x146 grid, 5x5 neighbourhood, filter after block 8) take the oracle several minutes each and run when
+SPV_SLOW_PARITY=1 is set; the oracle's free-running output is cached in tests/.oracle_cache (git-ignored),
+keyed by the configuration, the seeds and the oracle source, and holds nothing that came from the GPU."""
+import hashlib
+import json
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import synth
+from test_gpu_vit import _compare, ctx  # noqa: F401  (ctx is the module-scoped context fixture)
+
+pytestmark = pytest.mark.gpu
+SLOW = os.environ.get("SPV_SLOW_PARITY", "") == "1"
+CACHE = os.path.join(os.path.dirname(os.path.abspath(__file__)), ".oracle_cache")
+REPORT = os.environ.get("SPV_PARITY_REPORT", "")
+
+
+def _oracle_cached(full, w, image, gh, gw, key):
+    """Free-running oracle forward of a seeded configuration, cached on disk."""
+    src = open(os.path.join(os.path.dirname(oracle.__file__), "spv_oracle.c"), "rb").read()
+    h = hashlib.sha1(json.dumps(key, sort_keys=True).encode() + hashlib.sha1(src).digest()).hexdigest()[:20]
+    path = os.path.join(CACHE, h + ".npz")
+    if os.path.exists(path):
+        z = np.load(path)
+        kept_all = z["kept_all"] if "kept_all" in z.files else None
+        return {"out": z["out"], "kept_all": kept_all,
+                "kept_idx": None if kept_all is None else kept_all[:, kept_all.shape[1] - (z["out"].shape[1] - full["n_global"]):]}
+    r = oracle.vit_forward(full, w, image, gh, gw)
+    os.makedirs(CACHE, exist_ok=True)
+    if r["kept_all"] is None:
+        np.savez(path, out=r["out"])
+    else:
+        np.savez(path, out=r["out"], kept_all=r["kept_all"])
+    return r
+
+
+def _run(ctx, arch, cfg, grid, wseed, iseed, side, name, background=None, background_range=None):
+    w = synth.vit_weights(wseed, arch, grid, grid)
+    kw = {} if background_range is None else {"background_range": background_range}
+    if background is not None:
+        kw["background"] = background
+    image = synth.tissue_batch(iseed, 1, side, side, **kw)
+    full = dict(arch, **cfg)
+    key = dict(name=name, cfg={k: v for k, v in full.items()}, grid=grid, wseed=wseed, iseed=iseed, side=side, kw=kw)
+    report = {}
+    _compare(ctx, arch, cfg, grid, grid, 1, 0, w=w, image=image, report=report,
+             free_oracle=lambda: _oracle_cached(full, w, image, grid, grid, key))
+    if REPORT:
+        with open(REPORT, "a") as f:
+            f.write(json.dumps(dict(case=name, **report)) + "\n")
+    return report
+
+
+@pytest.mark.parametrize("mode", ["sparse_filter", "sparse", "dense"])
+def test_vitl16_1024_full_depth(ctx, mode):
+    """24 blocks, d 1024, 16 heads, MLP 4096 GELU, LayerScale; weights seed 2, image seed 3 (about 40 %
+    background); 8x8-patch blocks, 3x3 neighbourhood; filter after block 4 keeping 0.6."""
+    cfg = {"dense": dict(attn_mode=synth.ATTN_DENSE, block=8, radius=1),
+           "sparse": dict(attn_mode=synth.ATTN_SPARSE, block=8, radius=1),
+           "sparse_filter": dict(attn_mode=synth.ATTN_SPARSE, block=8, radius=1, filter_layer=4, keep_ratio=0.6)}[mode]
+    _run(ctx, synth.vit_l16(), cfg, 64, 2, 3, 1024, "vitl16_1024_" + mode, background=0.4)
+
+
+@pytest.mark.skipif(not SLOW, reason="several minutes of oracle time: set SPV_SLOW_PARITY=1")
+def test_vitl16_2048_benchmark_image(ctx):
+    """The first image of the default benchmark workload: 128x128 grid, filter after block 4 keeping 0.5."""
+    cfg = dict(attn_mode=synth.ATTN_SPARSE, block=8, radius=1, filter_layer=4, keep_ratio=0.5)
+    _run(ctx, synth.vit_l16(), cfg, 128, 2, 6, 2048, "vitl16_2048_sparse_filter", background_range=(0.3, 0.6))
+
+
+@pytest.mark.skipif(not SLOW, reason="about ten minutes of oracle time: set SPV_SLOW_PARITY=1")
+def test_vitg14_2044_full_depth(ctx):
+    """40 blocks, d 1536, 24 heads, SwiGLU 4096, patch 14, no LayerScale; 146x146 grid (19x19 blocks, the last
+    row and column 2 patches wide), 5x5 neighbourhood, filter after block 8 keeping 0.5; weights seed 4,
+    image seed 5 (about 50 % background)."""
+    cfg = dict(attn_mode=synth.ATTN_SPARSE, block=8, radius=2, filter_layer=8, keep_ratio=0.5)
+    _run(ctx, synth.vit_g14(), cfg, 146, 4, 5, 2044, "vitg14_2044_sparse_filter", background=0.5)
