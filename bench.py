@@ -52,6 +52,18 @@ WORKLOADS = {
 DEFAULT_WORKLOAD = "vitl16_2048_b4_sparse_filter"
 
 
+def config_of(wl, world):
+    a, c, g = wl["arch"], wl["cfg"], wl["grid"]
+    k = g * g
+    if c["filter_layer"] > 0:
+        k = int(np.ceil(c["keep_ratio"] * g * g - 1e-9))
+    return {"workload": wl["name"], "image": f"{wl['side']}x{wl['side']}", "batch_per_gpu": wl["batch"], "grid": f"{g}x{g}",
+            "tokens": a["n_global"] + g * g, "block": c["block"], "radius": c["radius"],
+            "filter_layer": c["filter_layer"], "keep_ratio": c["keep_ratio"], "kept": k,
+            "parallelism": "replicas" if world > 1 else "single GPU",
+            "l2": "inputs larger than L2 (activations of one step exceed 126 MB)"}
+
+
 def workload_config(name):
     arch_name, side, batch, block, radius, fl, keep, wseed, iseed = WORKLOADS[name]
     arch = synth.vit_l16() if arch_name == "l16" else synth.vit_g14()
@@ -253,7 +265,7 @@ def oracle_sample(wl, rows, seed=11):
 def run_reference(args, wl, rank):
     if rank != 0:
         return
-    rows = 512
+    rows = args.cpu_rows           # the same sample as the cpu_baseline leg of the GPU arm
     for _ in range(args.warmup):
         oracle_sample(wl, rows)
     times, rates, last = [], [], None
@@ -269,7 +281,7 @@ def run_reference(args, wl, rank):
         "impl": "reference", "metric": metric_name(wl), "value": value, "unit": "images/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl["name"], "l2": "inputs larger than L2"},
+        "config": config_of(wl, int(os.environ.get("WORLD_SIZE", "1"))),
         "cpu_baseline": {"value": value, "unit": "images/s", "cores": last["cores"], "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -364,6 +376,36 @@ def run_gpu(args, wl, rank, world):
     clocks = sampler.stop()
     peak_bytes = torch.cuda.max_memory_allocated()
 
+    # ---- the same steps with a spatially coherent kept set: random weights scatter the kept tokens over the
+    # blocks, the worst case for the block-sparse kernel; a trained backbone drops background.  forced_keep =
+    # the k darkest patches of each image (the tissue).
+    coh = None
+    if c["filter_layer"] > 0 and not args.quick:
+        fk_host = tissue_kept(img_host.numpy(), a["patch"], k)
+        fk = torch.from_numpy(fk_host).to(dev)
+        for _ in range(2):
+            ctx.vit_forward(c, dw, img, g, g, out=out, forced_keep=fk)
+        ctx.check()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        g0.record(stream)
+        for _ in range(args.steps):
+            ctx.vit_forward(c, dw, img, g, g, out=out, forced_keep=fk)
+        g1.record(stream)
+        barrier()
+        ms_coh = g0.elapsed_time(g1)
+        ctx.profile(True)
+        for _ in range(args.steps):
+            ctx.vit_forward(c, dw, img, g, g, out=out, forced_keep=fk)
+        prof_coh = ctx.profile_read()
+        ctx.profile(False)
+        ctx.check()
+        fl_coh = forward_flops(wl, fk_host)
+        coh = {"kept": "the k darkest patches of each image (tissue), given as forced_keep",
+               "images_per_s": B * args.steps / (ms_coh * 1e-3), "ms_per_step": ms_coh / args.steps,
+               "attn_patch_ms_per_step": prof_coh["attn_patch"]["ms"] / args.steps,
+               "attn_patch_useful_tflops": fl_coh["attn_patch"] * args.steps / (prof_coh["attn_patch"]["ms"] * 1e-3) / 1e12}
+
     # ---- end to end: pinned host images in, output tokens back to the host, every step.  The way a
     # user of the library would run a stream of batches: copies on their own streams, double-buffered,
     # so that the copy of batch i+1 and the read-back of batch i-1 overlap the forward of batch i.
@@ -447,11 +489,7 @@ def run_gpu(args, wl, rank, world):
         "metric": metric_name(wl), "value": value, "unit": "images/s", "n_gpus": world, "steps": steps, "warmup": n_warm,
         "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl["name"], "image": f"{side}x{side}", "batch_per_gpu": B, "grid": f"{g}x{g}",
-                   "tokens": a["n_global"] + g * g, "block": c["block"], "radius": c["radius"],
-                   "filter_layer": c["filter_layer"], "keep_ratio": c["keep_ratio"], "kept": k,
-                   "parallelism": "replicas" if world > 1 else "single GPU",
-                   "l2": "inputs larger than L2 (activations of one step exceed 126 MB)"},
+        "config": config_of(wl, world),
         "clocks": clocks, "gpu_launches": launches,
         "e2e": {"value": images / (ms_e2e * 1e-3), "unit": "images/s",
                 "h2d_bytes_per_step": img_host.numel() * 4, "d2h_bytes_per_step": out_host.numel() * 2},
@@ -459,6 +497,9 @@ def run_gpu(args, wl, rank, world):
         "useful_tflops": total_flops * steps * world / (ms * 1e-3) / 1e12,
         "peak_hbm_bytes": peak_bytes,
     }
+    if coh is not None:
+        coh["attn_patch_frac"] = coh["attn_patch_useful_tflops"] / pk["tensor"]
+        line["coherent_kept"] = coh
     if world == 1 and not args.no_cpu and not args.quick:
         cb = oracle_sample(wl, args.cpu_rows)
         line["cpu_baseline"] = {
@@ -482,11 +523,22 @@ def coherent_kept(seed, grid, keep):
     rng = np.random.Generator(np.random.PCG64(seed))
     n = grid * grid
     k = int(np.ceil(keep * n - 1e-9))
-    bg = synth.background_mask(rng, grid, grid, 1.0 - k / n).reshape(-1)
+    bg = synth.background_mask(rng, grid, grid, 1.0 - k / n, cell=32).reshape(-1)   # regions a few blocks wide
     kept = np.flatnonzero(~bg)[:k]
     if kept.size < k:
         kept = np.sort(np.concatenate([kept, np.flatnonzero(bg)[:k - kept.size]]))
     return kept.astype(np.int32)
+
+
+def tissue_kept(images, patch, k):
+    """[B, k] ascending positions of the k darkest patches of each image (mean of the green channel; ties to the
+    lower index): on these images that is the tissue, i.e. the spatially coherent set a trained backbone's CLS
+    scores would keep (Sec. 3.3 reports that the pruned tokens are background).  images: fp32 [B, 3, S, S]."""
+    B, _, S, _ = images.shape
+    g = S // patch
+    m = images[:, 1].reshape(B, g, patch, g, patch).mean(axis=(2, 4)).reshape(B, g * g)
+    order = np.argsort(m, axis=1, kind="stable")[:, :k]
+    return np.sort(order, axis=1).astype(np.int32)
 
 
 def block_major(pos, grid, block):
@@ -787,7 +839,8 @@ def run_ablation(args):
     points += [("radius", r, dict(radius=r)) for r in (0, 1, 2, 3)]
     points += [("n_global", G, dict(G=G)) for G in (1, 5, 9)]
     points += [("filters", "4:0.7,12:0.7", dict(filters=[(4, 0.7), (12, 0.7)])),
-               ("filters", "4:0.5", dict(filters=[(4, 0.5)]))]
+               ("filters", "4:0.5", dict(filters=[(4, 0.5)])),
+               ("unfused_filter", 1, dict(unfused=1)), ("unfused_filter", 0, dict(unfused=0))]
     weights = {}
     for axis, val, o in points:
         G = o.get("G", 1)
@@ -798,7 +851,8 @@ def run_ablation(args):
             weights[G] = ctx.make_vit_weights(synth.vit_weights(2, arch, g, g))
         dw = weights[G]
         stages = o.get("filters", [(4, o.get("keep", 0.5))])
-        cfg = dict(arch, attn_mode=synth.ATTN_SPARSE, block=o.get("block", 8), radius=o.get("radius", 1), filters=stages)
+        cfg = dict(arch, attn_mode=synth.ATTN_SPARSE, block=o.get("block", 8), radius=o.get("radius", 1), filters=stages,
+                   unfused_filter=o.get("unfused", 0))
         wl = dict(name="ablation", arch=arch, cfg=dict(cfg, filter_layer=stages[0][0], keep_ratio=stages[0][1]),
                   side=side, grid=g, batch=B)
         kept = None
@@ -847,7 +901,9 @@ def run_ablation(args):
                           "images_per_s": B / (ms * 1e-3), "attn_patch_ms_per_step": attn_ms,
                           "attn_useful_tflops": flop / (attn_ms * 1e-3) / 1e12,
                           "attn_frac_of_sustained_bf16": flop / (attn_ms * 1e-3) / 1e12 / pk["tensor"],
-                          "gemm_ms_per_step": prof["gemm"]["ms"] / steps, "steps": steps}), flush=True)
+                          "gemm_ms_per_step": prof["gemm"]["ms"] / steps,
+                          "filter_select_ms_per_step": prof["filter_select"]["ms"] / steps,
+                          "attn_global_ms_per_step": prof["attn_global"]["ms"] / steps, "steps": steps}), flush=True)
 
 
 # --------------------------------------------------------------------------------------------
@@ -915,7 +971,7 @@ def main():
     ap.add_argument("--sweep-ablation", action="store_true",
                     help="keep ratio / block / radius / global tokens / two filter stages, one JSON line per point")
     ap.add_argument("--ablation-side", type=int, default=2048)
-    ap.add_argument("--cpu-rows", type=int, default=16384, help="rows of the CPU-oracle sample")
+    ap.add_argument("--cpu-rows", type=int, default=8192, help="rows of the CPU-oracle sample (both arms)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--quick", action="store_true",
                     help="profiling aid: exactly --warmup warm-up steps, no end-to-end and no CPU leg")

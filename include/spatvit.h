@@ -207,6 +207,10 @@ typedef struct {
                              keep_ratios[i] in (0, 1]; filter_layer / keep_ratio are ignored      */
   int32_t filter_layers[SPV_MAX_FILTERS];
   double keep_ratios[SPV_MAX_FILTERS];
+  int32_t unfused_filter; /* 0 (default): the CLS->patch weights are evaluated, averaged over the heads
+                             and turned into ranking keys in one kernel; 1: the score tensor
+                             [batch, heads, patches] is written first and then averaged (the two
+                             standalone steps).  Same kept set either way                        */
 } spv_vit_config;
 
 /* Per-layer weights: matrices bf16 [out_features, in_features] row-major; vectors fp32. */

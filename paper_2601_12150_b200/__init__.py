@@ -52,7 +52,8 @@ class VitConfig(C.Structure):
                 ("n_global", C.c_int32), ("has_layerscale", C.c_int32), ("ln_eps", C.c_float),
                 ("attn_mode", C.c_int32), ("block", C.c_int32), ("radius", C.c_int32),
                 ("filter_layer", C.c_int32), ("keep_ratio", C.c_double),
-                ("n_filters", C.c_int32), ("filter_layers", C.c_int32 * 4), ("keep_ratios", C.c_double * 4)]
+                ("n_filters", C.c_int32), ("filter_layers", C.c_int32 * 4), ("keep_ratios", C.c_double * 4),
+                ("unfused_filter", C.c_int32)]
 
 
 LAYER_FIELDS = ["ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_o", "b_o", "ls1", "ln2_g", "ln2_b",
@@ -378,7 +379,7 @@ class Context:
                       cfg["patch"], cfg["n_global"], cfg.get("has_layerscale", 0), cfg.get("ln_eps", 1e-6),
                       cfg["attn_mode"], cfg.get("block", 8), cfg.get("radius", 1),
                       0 if multi else cfg.get("filter_layer", 0), 1.0 if multi else cfg.get("keep_ratio", 1.0),
-                      len(stages) if multi else 0, fl, kr)
+                      len(stages) if multi else 0, fl, kr, int(cfg.get("unfused_filter", 0)))
         B = image.shape[0]
         npatch = grid_h * grid_w
         counts, cur = [], npatch

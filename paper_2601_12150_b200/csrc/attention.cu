@@ -12,11 +12,14 @@
 //   attn_plan_*        per-block token counts (binary search in the sorted positions), scan,
 //                      each block row cut into 128-row query tiles
 //   attn_regroup       row-major -> block-major copy of Q, K, V (only for row-major callers)
-//   attn_patch_kernel  flash-style tcgen05 kernel: S = Q K^T into TMEM, online softmax by 128
-//                      row-owning threads, P written back to TMEM as bf16, O += P V with V as an
-//                      MN-major shared-memory operand; the global tokens' keys and values join
-//                      the softmax state in the epilogue (dot products on the CUDA cores while
-//                      the last P V runs), so key tiles stay multiples of the MMA shape
+//   attn_patch_kernel  flash-style tcgen05 kernel: S = Q K^T of a 128-row query tile and a 32-key tile into
+//                      one of three TMEM buffers, online softmax by 128 row-owning threads whose four warps
+//                      advance independently (a warp whose rows have no key in a tile writes P = 0 and moves
+//                      on; warps meet only when O has to be rescaled), P written over its own S as bf16,
+//                      O += P V with V as an MN-major shared-memory operand; Q K^T is issued by two threads
+//                      (even / odd key tiles), P V by one; the global tokens' keys and values join the softmax state in the epilogue
+//                      (dot products on the CUDA cores while the last P V runs), so key tiles stay multiples
+//                      of the MMA shape
 //   attn_global_*      the dense rows of the global (CLS) queries and the CLS->patch scores
 #include "attention.cuh"
 
@@ -25,23 +28,25 @@ namespace {
 using namespace spv;
 
 constexpr int TQ = 128;            // query rows per tile (MMA M)
-constexpr int TK = 64;             // keys per tile (MMA N of S, K extent of P V): with 64, a CTA needs 160 TMEM
-                                   // columns and 136 registers per softmax thread, so three CTAs fit an SM
+constexpr int TK = 32;             // keys per tile (MMA N of S, K extent of P V): three S buffers of 32 columns and
+                                   // O make 160 TMEM columns, so three CTAs fit an SM
 constexpr int HD = 64;             // head_dim
-constexpr int KST = 3;             // K / V smem stages
-constexpr int ATT_THREADS = 256;   // warps 0-3 softmax (one warpgroup), 4 TMA, 5 MMA, 6-7 idle: the second
-                                   // warpgroup exists so that it can hand its registers to the first
+constexpr int KST = 6;             // K / V smem stages (Q K^T runs up to two key tiles ahead of P V)
+constexpr int NSB = 3;             // S / P buffers in TMEM: a softmax warp may be two key tiles ahead of the slowest
+constexpr int ATT_THREADS = 256;   // warps 0-3 softmax (one warpgroup), 4 TMA, 5-7 MMA issue: the second warpgroup
+                                   // hands most of its registers to the first
 constexpr int TILE_BYTES = 128 * 128;  // Q tile
 constexpr int KV_BYTES = TK * 128;      // K or V tile
 constexpr int MAXG = 16;           // global tokens
 // Shared memory of a CTA for `grows` rows of global tokens (8 or 16: with up to 8, three CTAs fit an SM):
 // Q tile, K / V stages, the global tokens' key and value rows (128 B each), barriers, their scores per query row.
 constexpr int att_smem(int grows) {
-  return TILE_BYTES + 2 * KST * KV_BYTES + 2 * grows * 128 + 1024 /*align*/ + 256 /*barriers*/ + grows * 128 * 4;
+  return TILE_BYTES + 2 * KST * KV_BYTES + 2 * grows * 128 + 1024 /*align*/ + 512 /*barriers*/ + grows * 128 * 4;
 }
-// two TMEM allocations per CTA, 160 columns in all, so that three CTAs share an SM's 512
-constexpr uint32_t TMEM_COLS = 128, TMEM_P_COLS = 32;
-constexpr uint32_t S_COL = 0, O_COL = 64;
+// two TMEM allocations per CTA, 160 columns in all, so that three CTAs share an SM's 512: O and two S buffers in
+// the first, the third S buffer in the second.  A row's P (bf16, 16 columns) is written over its own S.
+constexpr uint32_t TMEM_COLS = 128, TMEM_S2_COLS = 32;
+constexpr uint32_t O_COL = 0, S_COL = 64;
 
 // ------------------------------------------------------------------------------------------
 // plan
@@ -293,13 +298,13 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   uint64_t* k_empty = k_full + KST;
   uint64_t* v_full = k_empty + KST;
   uint64_t* v_empty = v_full + KST;
-  uint64_t* s_full = v_empty + KST;
-  uint64_t* s_free = s_full + 1;
-  uint64_t* p_full = s_free + 1;
-  uint64_t* pv_done = p_full + 1;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + 1);
-  volatile uint32_t* abort_flag = tmem_slot + 1;
-  float* s_sg = reinterpret_cast<float*>(bars + 32);     // [G][128] scaled scores of the global keys
+  uint64_t* s_full = v_empty + KST;      // [NSB] Q K^T of the buffer's key tile has completed
+  uint64_t* p_full = s_full + NSB;       // [NSB] all 128 rows have written P (and read S) of the buffer
+  uint64_t* pv_done = p_full + NSB;      // [NSB] P V of the buffer's key tile (and all before it) has completed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + NSB);
+  volatile uint32_t* abort_flag = tmem_slot + 3;
+  float* s_sg = reinterpret_cast<float*>(bars + 64);     // [G][128] scaled scores of the global keys
+  static_assert(1 + 4 * KST + 3 * NSB + 2 <= 64, "barrier area");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = p.radius, G = p.n_global;
@@ -313,25 +318,24 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
       mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
     }
-    mbar_init(s_full, 1);
-    mbar_init(s_free, 128);
-    mbar_init(p_full, 128);
-    mbar_init(pv_done, 1);
+    for (int s = 0; s < NSB; ++s) { mbar_init(&s_full[s], 1); mbar_init(&p_full[s], 128); mbar_init(&pv_done[s], 1); }
     *abort_flag = 0;
     mbar_fence_init();
   }
   if (warp == 5) {
     tmem_alloc(tmem_slot, TMEM_COLS);
-    tmem_alloc(tmem_slot + 2, TMEM_P_COLS);
+    tmem_alloc(tmem_slot + 2, TMEM_S2_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot, tmem_p = tmem_slot[2];
+  const uint32_t tmem = *tmem_slot, tmem_s2 = tmem_slot[2];
+  // S buffer b of the three: two sit behind O in the first allocation, the third is the second allocation
+  auto s_col = [&](uint32_t buf) { return buf < 2 ? tmem + S_COL + buf * TK : tmem_s2; };
 
-  // the softmax warpgroup holds a whole score row of the key tile (64 columns) per thread; the other warpgroup
-  // needs few registers
+  // the softmax warpgroup holds a score row of the key tile per thread; the other warpgroup needs few
+  // registers (the kernel starts with 80 per thread: 80 + (80 - 24) = 136)
   if (warp >= 4) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 24;");
   if (warp == 4) {
@@ -357,43 +361,53 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
       }
     }
-  } else if (warp == 5) {
-    // ---------------- MMA issuer
+  } else {
+    // ---------------- MMA issuers.  One thread gets a tcgen05.mma of these small shapes issued only about every
+    // 120 cycles (measured): S = Q K^T has two issuing threads (warp 5 the even key tiles, warp 7 the odd ones;
+    // consecutive tiles go to different S buffers) and O += P V one (warp 6; its instructions accumulate into the
+    // same O and stay in one thread's order).
     if (lane == 0) {
       uint32_t n_kv = 0;
       for (int cy = cy0; cy <= cy1; ++cy) {
         const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
         n_kv += (uint32_t)((ke - ks + TK - 1) / TK);
       }
-      constexpr uint32_t idesc_s = idesc_bf16(TQ, TK, false);
-      constexpr uint32_t idesc_o = idesc_bf16(TQ, HD, true);
-      const uint64_t dq = smem_desc_sw128(smem_u32(sQ));
-      auto issue_qk = [&](uint32_t j) {
-        const int s = j % KST;
-        mbar_wait(&k_full[s], (j / KST) & 1, abort_flag, p.status, 0x1300 + s);
-        if (j > 0) mbar_wait(s_free, (j - 1) & 1, abort_flag, p.status, 0x1400);
-        tc_fence_after();
-        const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * KV_BYTES));
+      if (warp != 6) {
+        constexpr uint32_t idesc_s = idesc_bf16(TQ, TK, false);
+        const uint64_t dq = smem_desc_sw128(smem_u32(sQ));
+        mbar_wait(q_full, 0, abort_flag, p.status, 0x1000);
+        // Q K^T of key tile t goes to S buffer t % 3, up to two tiles ahead of the softmax, as soon as P V of
+        // tile t - 3, which read its P from that buffer, has completed
+        for (uint32_t t = warp == 5 ? 0 : 1; t < n_kv; t += 2) {
+          const int s = t % KST;
+          const uint32_t sb = t % NSB;
+          mbar_wait(&k_full[s], (t / KST) & 1, abort_flag, p.status, 0x1300 + s);
+          if (t >= NSB) mbar_wait(&pv_done[sb], ((t - NSB) / NSB) & 1, abort_flag, p.status, 0x1400 + sb);
+          tc_fence_after();
+          const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * KV_BYTES));
+          const uint32_t d_s = s_col(sb);
 #pragma unroll
-        for (int kk = 0; kk < HD / 16; ++kk)
-          mma_ss(tmem + S_COL, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_s, kk != 0);
-        tc_commit(s_full);
-        tc_commit(&k_empty[s]);
-      };
-      mbar_wait(q_full, 0, abort_flag, p.status, 0x1000);
-      if (n_kv > 0) issue_qk(0);
-      for (uint32_t j = 0; j < n_kv; ++j) {
-        if (j + 1 < n_kv) issue_qk(j + 1);
-        const int s = j % KST;
-        mbar_wait(&v_full[s], (j / KST) & 1, abort_flag, p.status, 0x1500 + s);
-        mbar_wait(p_full, j & 1, abort_flag, p.status, 0x1600);
-        tc_fence_after();
-        const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * KV_BYTES));
+          for (int kk = 0; kk < HD / 16; ++kk)
+            mma_ss(d_s, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_s, kk != 0);
+          tc_commit(&s_full[sb]);
+          tc_commit(&k_empty[s]);
+        }
+      } else {
+        constexpr uint32_t idesc_o = idesc_bf16(TQ, HD, true);
+        for (uint32_t j = 0; j < n_kv; ++j) {
+          const int s = j % KST;
+          const uint32_t sb = j % NSB;
+          mbar_wait(&v_full[s], (j / KST) & 1, abort_flag, p.status, 0x1500 + s);
+          mbar_wait(&p_full[sb], (j / NSB) & 1, abort_flag, p.status, 0x1600 + sb);
+          tc_fence_after();
+          const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * KV_BYTES));
+          const uint32_t a_p = s_col(sb);
 #pragma unroll
-        for (int kk = 0; kk < TK / 16; ++kk)
-          mma_ts(tmem + O_COL, tmem_p + kk * 8, dv + (uint64_t)(kk * 128), idesc_o, (j | kk) != 0);
-        tc_commit(pv_done);
-        tc_commit(&v_empty[s]);
+          for (int kk = 0; kk < TK / 16; ++kk)
+            mma_ts(tmem + O_COL, a_p + kk * 8, dv + (uint64_t)(kk * 128), idesc_o, (j | kk) != 0);
+          tc_commit(&pv_done[sb]);
+          tc_commit(&v_empty[s]);
+        }
       }
     }
   }
@@ -403,8 +417,8 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int row = threadIdx.x;
     const int tok = q_begin + row;
     const bool valid = tok < q_end;
-    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-    const uint32_t lane_addr_p = tmem_p + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const uint32_t lane_addr = tmem + lane_off;
     int bxq = bx_first;
     if (valid) bxq = __ldg(p.tok_blk + (size_t)b * p.n_patch + tok) % p.nbx;
     const int rlo = max(bxq - r, 0), rhi = min(bxq + r, p.nbx - 1);
@@ -427,109 +441,91 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const bool v0 = __shfl_sync(0xffffffffu, (int)valid, 0) != 0;
         if (!valid) { lo = lo0; hi = v0 ? hi0 : lo0; }
       }
+      // over the warp's rows: a superset of the union of the allowed ranges (keys outside it are not even
+      // read) and a subset of their intersection (keys inside it need no mask), once per block row
+      const int ulo = __reduce_min_sync(0xffffffffu, lo), uhi = __reduce_max_sync(0xffffffffu, hi);
+      const int ilo = __reduce_max_sync(0xffffffffu, lo), ihi = __reduce_min_sync(0xffffffffu, hi);
       for (int kb = ks; kb < ke; kb += TK, ++j) {
-        // this row's allowed keys are the tile columns [c_lo, c_hi); u_* is the union over the
-        // warp's rows (columns outside it are not even read), i_* the intersection (columns
-        // inside it need no per-element mask)
-        const int c_lo = min(max(lo - kb, 0), TK), c_hi = min(max(hi - kb, 0), TK);
-        const bool some = c_lo < c_hi;
-        const int u_lo = __reduce_min_sync(0xffffffffu, some ? c_lo : TK);
-        const int u_hi = __reduce_max_sync(0xffffffffu, some ? c_hi : 0);
-        const int i_lo = __reduce_max_sync(0xffffffffu, some ? c_lo : TK);
-        const int i_hi = __reduce_min_sync(0xffffffffu, some ? c_hi : 0);
-        mbar_wait(s_full, j & 1, abort_flag, p.status, 0x1800);
+        const uint32_t sbuf = j % NSB, sph = (j / NSB) & 1;
+        const uint32_t s_addr = s_col(sbuf) + lane_off;
+        mbar_wait(&s_full[sbuf], sph, abort_flag, p.status, 0x1800 + sbuf);
         tc_fence_after();
-        // one pass: the live 32-column chunks of S go to registers, then S is released
-        uint32_t sr[TK];
+        if (uhi <= kb || ulo >= kb + TK) {
+          // no row of this warp has a key in the tile: P = 0 for its 32 rows and on to the next tile, without
+          // waiting for the other warps (their rows' P V needs this warp's rows of P all the same)
+          uint32_t z[16];
 #pragma unroll
-        for (int c = 0; c < TK / 32; ++c)
-          if (32 * c < u_hi && 32 * c + 32 > u_lo) tmem_ld32(lane_addr + S_COL + 32 * c, sr + 32 * c);
+          for (int i = 0; i < 16; ++i) z[i] = 0u;
+          tmem_st16(s_addr, z);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(&p_full[sbuf]);
+          continue;
+        }
+        uint32_t sr[TK];
+        tmem_ld32(s_addr, sr);
         tc_wait_ld();
-        tc_fence_before();
-        mbar_arrive(s_free);                               // S may be overwritten by the next Q K^T
-        // boundary chunks (some of the warp's rows see only part of them) are masked in registers:
-        // column c is allowed iff c_lo <= c < c_hi, one unsigned compare; chunks inside the
-        // intersection of the warp's rows skip this
-        {
+        // a tile that is not inside every row's range is masked in registers: column c is allowed iff
+        // c_lo <= c < c_hi, one unsigned compare
+        if (!(kb >= ilo && kb + TK <= ihi)) {
+          const int c_lo = min(max(lo - kb, 0), TK), c_hi = min(max(hi - kb, 0), TK);
           const uint32_t width = (uint32_t)(c_hi - c_lo);
 #pragma unroll
-          for (int c = 0; c < TK / 32; ++c) {
-            if (32 * c < u_hi && 32 * c + 32 > u_lo && !(32 * c >= i_lo && 32 * c + 32 <= i_hi)) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if ((uint32_t)(32 * c + i - c_lo) >= width) sr[32 * c + i] = 0xff800000u;
-            }
-          }
+          for (int i = 0; i < TK; ++i)
+            if ((uint32_t)(i - c_lo) >= width) sr[i] = 0xff800000u;
         }
-        float mx = -INFINITY;
+        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < TK / 32; ++c) {
-          if (32 * c < u_hi && 32 * c + 32 > u_lo) {
-            float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
-#pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              m0 = fmax3(m0, __uint_as_float(sr[32 * c + i]), __uint_as_float(sr[32 * c + i + 1]));
-              m1 = fmax3(m1, __uint_as_float(sr[32 * c + i + 2]), __uint_as_float(sr[32 * c + i + 3]));
-              m2 = fmax3(m2, __uint_as_float(sr[32 * c + i + 4]), __uint_as_float(sr[32 * c + i + 5]));
-              m3 = fmax3(m3, __uint_as_float(sr[32 * c + i + 6]), __uint_as_float(sr[32 * c + i + 7]));
-            }
-            mx = fmax3(mx, fmaxf(m0, m1), fmaxf(m2, m3));
-          }
+        for (int i = 0; i < TK; i += 8) {
+          m0 = fmax3(m0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+          m1 = fmax3(m1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+          m2 = fmax3(m2, __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
+          m3 = fmax3(m3, __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
         }
+        const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
         // lazy rescale: the running maximum only moves when it would grow by more than 2^8
         const float m_t = mx * sl2;
         const bool need = m_t > m + 8.0f;
         const float m_new = need ? m_t : m;
         const float alpha = need ? fast_exp2(m - m_new) : 1.0f;
-        const bool any_need = __any_sync(0xffffffffu, need);
-        if (j > 0) {
-          mbar_wait(pv_done, (j - 1) & 1, abort_flag, p.status, 0x1900);   // P buffer and O are free
+        // O has to be rescaled only where something has been accumulated (l > 0); that is the one place where a
+        // warp waits for the P V of the previous key tile, i.e. for the other warps
+        if (__any_sync(0xffffffffu, need && l > 0.f)) {
+          const uint32_t pj = j - 1;                       // l > 0 implies j > 0
+          mbar_wait(&pv_done[pj % NSB], (pj / NSB) & 1, abort_flag, p.status, 0x1900);
           tc_fence_after();
-          if (any_need) {
 #pragma unroll
-            for (int c = 0; c < HD / 32; ++c) {
-              uint32_t orr[32];
-              tmem_ld32(lane_addr + O_COL + 32 * c, orr);
-              tc_wait_ld();
+          for (int c = 0; c < HD / 32; ++c) {
+            uint32_t orr[32];
+            tmem_ld32(lane_addr + O_COL + 32 * c, orr);
+            tc_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-              tmem_st32(lane_addr + O_COL + 32 * c, orr);
-            }
+            for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+            tmem_st32(lane_addr + O_COL + 32 * c, orr);
           }
         }
-        // p = 2^(s*scale - m) chunk by chunk, packed to bf16 pairs and written to TMEM at once
-        // (masked scores are -inf, so p = 0)
-        // (two scores per packed fp32x2 multiply-add and per packed add)
+        // p = 2^(s*scale - m), packed to bf16 pairs and written over the first half of this row's S (masked
+        // scores are -inf, so p = 0); two scores per packed fp32x2 multiply-add and add
         float2 rs_a = make_float2(0.f, 0.f), rs_b = make_float2(0.f, 0.f);
         const float2 sl2_2 = make_float2(sl2, sl2), nm_2 = make_float2(-m_new, -m_new);
+        uint32_t pk[16];
 #pragma unroll
-        for (int c = 0; c < TK / 32; ++c) {
-          uint32_t pk[16];
-          if (32 * c < u_hi && 32 * c + 32 > u_lo) {
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(sr[32 * c + i]), __uint_as_float(sr[32 * c + i + 1])),
-                                           sl2_2, nm_2);
-              const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(sr[32 * c + i + 2]), __uint_as_float(sr[32 * c + i + 3])),
-                                           sl2_2, nm_2);
-              const float2 p0 = make_float2(fast_exp2(x0.x), fast_exp2(x0.y));
-              const float2 p1 = make_float2(fast_exp2(x1.x), fast_exp2(x1.y));
-              rs_a = __fadd2_rn(rs_a, p0);
-              rs_b = __fadd2_rn(rs_b, p1);
-              pk[i / 2] = pack_bf16(p0.x, p0.y);
-              pk[i / 2 + 1] = pack_bf16(p1.x, p1.y);
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) pk[i] = 0u;
-          }
-          tmem_st16(lane_addr_p + 16 * c, pk);
+        for (int i = 0; i < TK; i += 4) {
+          const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), sl2_2, nm_2);
+          const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3])), sl2_2, nm_2);
+          const float2 p0 = make_float2(fast_exp2(x0.x), fast_exp2(x0.y));
+          const float2 p1 = make_float2(fast_exp2(x1.x), fast_exp2(x1.y));
+          rs_a = __fadd2_rn(rs_a, p0);
+          rs_b = __fadd2_rn(rs_b, p1);
+          pk[i / 2] = pack_bf16(p0.x, p0.y);
+          pk[i / 2 + 1] = pack_bf16(p1.x, p1.y);
         }
+        tmem_st16(s_addr, pk);
         l = l * alpha + ((rs_a.x + rs_a.y) + (rs_b.x + rs_b.y));
         m = m_new;
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(p_full);
+        mbar_arrive(&p_full[sbuf]);
       }
     }
     // ---------------- epilogue: the global tokens join the softmax, then O / l
@@ -567,7 +563,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     for (int g = 0; g < G; ++g) l_f += fast_exp2(s_sg[g * 128 + row] - m_f);
     const float inv = 1.0f / l_f;
     if (j > 0) {
-      mbar_wait(pv_done, (j - 1) & 1, abort_flag, p.status, 0x1A00);
+      mbar_wait(&pv_done[(j - 1) % NSB], ((j - 1) / NSB) & 1, abort_flag, p.status, 0x1A00);
       tc_fence_after();
     }
     float of[HD];
@@ -649,7 +645,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   tc_fence_after();
   if (warp == 5) {
     tmem_dealloc(tmem, TMEM_COLS);
-    tmem_dealloc(tmem_p, TMEM_P_COLS);
+    tmem_dealloc(tmem_s2, TMEM_S2_COLS);
   }
 }
 
@@ -787,7 +783,8 @@ __global__ void __launch_bounds__(256) attn_global_combine(const float* __restri
                                                            int n_tok, int n_global, int heads,
                                                            __nv_bfloat16* __restrict__ o, int64_t o_sb,
                                                            int64_t o_st, int64_t o_sh, float* __restrict__ scores,
-                                                           const int32_t* __restrict__ score_idx, int score_stride) {
+                                                           const int32_t* __restrict__ score_idx, int score_stride,
+                                                           float* __restrict__ head_stats) {
   __shared__ float s_m, s_l;
   __shared__ float s_red[16];
   const int h = blockIdx.x, bg = blockIdx.y;
@@ -825,6 +822,12 @@ __global__ void __launch_bounds__(256) attn_global_combine(const float* __restri
     for (int c = 0; c < n_chunks; ++c)
       acc += part_o[(pbase + c) * HD + threadIdx.x] * __expf(part_ml[(pbase + c) * 2] - M);
     o[b * o_sb + (int64_t)g * o_st + (int64_t)h * o_sh + threadIdx.x] = __float2bfloat16(acc * inv);
+  }
+  // (row maximum of the scaled logits, 1 / row sum) of global token 0: with the logits they give the softmax
+  // weights to a consumer that folds them into its own pass (the fused ranking of the token filter)
+  if (head_stats && g == 0 && threadIdx.x == 0) {
+    head_stats[((size_t)b * heads + h) * 2] = M;
+    head_stats[((size_t)b * heads + h) * 2 + 1] = inv;
   }
   if (scores && g == 0) {
     const float* lg = logits + ((size_t)bg * heads + h) * n_tok;
@@ -954,7 +957,7 @@ size_t spv_attn_global_bytes(int32_t batch, int32_t n_global, int32_t heads, int
 
 int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, float* scores,
                              const int32_t* score_idx, int32_t score_stride, void* ws, size_t ws_bytes,
-                             cudaStream_t stream) {
+                             cudaStream_t stream, float* head_stats, const float** logits_out) {
   const int n_tok = plan->n_global + plan->n_patch, G = plan->n_global, B = plan->batch;
   if (ws_bytes < spv_attn_global_bytes(B, G, io->heads, n_tok)) return SPV_ERR_WORKSPACE;
   const size_t rows = (size_t)B * G * io->heads;
@@ -969,7 +972,8 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   float* part_ml = (float*)w; w += spv_align_up(rows * chunks * 2 * 4, 256);
   float* part_o = (float*)w;
   SpvProfScope prof(ctx, SPV_K_ATTN_GLOBAL, stream);
-  if (scores) attn_global_partial<true><<<dim3(io->heads, chunks, B * G), 256, 0, stream>>>(
+  if (logits_out) *logits_out = logits;
+  if (scores || head_stats) attn_global_partial<true><<<dim3(io->heads, chunks, B * G), 256, 0, stream>>>(
       (const __nv_bfloat16*)io->q, (const __nv_bfloat16*)io->k, (const __nv_bfloat16*)io->v, io->sb, io->st, io->sh,
       n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks, chunk_len);
   else attn_global_partial<false><<<dim3(io->heads, chunks, B * G), 256, 0, stream>>>(
@@ -977,7 +981,8 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
       n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks, chunk_len);
   attn_global_combine<<<dim3(io->heads, B * G), 256, 0, stream>>>(logits, part_ml, part_o, chunks, n_tok, G,
                                                                  io->heads, (__nv_bfloat16*)io->o, io->o_sb,
-                                                                 io->o_st, io->o_sh, scores, score_idx, score_stride);
+                                                                 io->o_st, io->o_sh, scores, score_idx, score_stride,
+                                                                 head_stats);
   return spv_launch_ok(ctx, 2);
 }
 

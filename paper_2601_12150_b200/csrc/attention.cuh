@@ -48,6 +48,9 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
 // (NULL = t); score_stride >= the largest index + 1 (the patch count, or the grid size when the indices
 // are original positions).
 size_t spv_attn_global_bytes(int32_t batch, int32_t n_global, int32_t heads, int32_t n_tok);
+// head_stats (optional): fp32 [B][heads][2] = (row maximum of the scaled logits, 1 / row sum) of global token 0;
+// logits_out then receives the scaled logits [B*G][heads][n_tok] inside `ws` (valid until `ws` is written again):
+// weight of token t = exp(logit[t] - maximum) / sum, which the fused ranking of the token filter evaluates itself.
 int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, float* scores,
                              const int32_t* score_idx, int32_t score_stride, void* ws, size_t ws_bytes,
-                             cudaStream_t stream);
+                             cudaStream_t stream, float* head_stats = nullptr, const float** logits_out = nullptr);

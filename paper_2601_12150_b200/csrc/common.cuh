@@ -29,6 +29,7 @@ struct spv_ctx {
   int32_t prof_on;
   // one-time per-device launch configuration (function attributes are per device, and a context is bound to one)
   int32_t attn_configured;
+  int32_t attn_ctas_per_sm[2];   // resident CTAs of the attention kernel per SM: up to 8 / up to 16 global tokens
   int32_t gemm_single_configured[8];   // per epilogue variant
   int32_t gemm_max_pairs[8];     // per epilogue variant: CTA pairs of the pair-form GEMM that can be resident at
                                  // once (0 = not yet queried)

@@ -42,6 +42,32 @@ __global__ void __launch_bounds__(256) filter_mean_key(const float* __restrict__
   if (mean_out) mean_out[(size_t)b * n_patch + j] = mean;
 }
 
+// The same head mean and key, with the softmax weight of every head evaluated here from the global row's
+// scaled logits: p = exp(logit - max_h) * inv_sum_h, summed in head order.  One thread per present patch; the
+// mean and key land at the patch's original position (keys of absent positions were zeroed beforehand).
+__global__ void __launch_bounds__(256) filter_mean_key_logits(const float* __restrict__ logits,
+                                                              const float* __restrict__ head_stats, int heads,
+                                                              int n_global, int n_tok,
+                                                              const int32_t* __restrict__ cur_pos, int npad,
+                                                              float* __restrict__ mean_ws,
+                                                              uint32_t* __restrict__ key_ws) {
+  const int b = blockIdx.y;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n_cur = n_tok - n_global;
+  if (t >= n_cur) return;
+  const float* lg = logits + (size_t)b * n_global * heads * n_tok + n_global + t;
+  const float* hs = head_stats + (size_t)b * heads * 2;
+  float sum = 0.0f;
+  for (int h = 0; h < heads; ++h) {
+    const float p = __expf(__ldg(lg + (size_t)h * n_tok) - __ldg(hs + 2 * h)) * __ldg(hs + 2 * h + 1);
+    sum = __fadd_rn(sum, p);
+  }
+  const float mean = __fdiv_rn(sum, (float)heads);
+  const int pos = cur_pos ? __ldg(cur_pos + (size_t)b * n_cur + t) : t;
+  mean_ws[(size_t)b * npad + pos] = mean;
+  key_ws[(size_t)b * npad + pos] = rank_key(mean);
+}
+
 // Block-wide exclusive scan of two counters; returns this thread's exclusive prefixes and the
 // block totals.  Called by all kSelThreads threads.
 __device__ __forceinline__ void block_scan2(int a, int b, int& ea, int& eb, int& ta, int& tb, int (*warp_tot)[2]) {
@@ -269,6 +295,28 @@ int32_t spv_filter_run_k(spv_ctx* ctx, const spv_filter_desc* d, int32_t k, cons
     ++launches;
   }
   return spv_launch_ok(ctx, launches);
+}
+
+int32_t spv_filter_rank_logits(spv_ctx* ctx, int32_t batch, int32_t heads, int32_t n_global, int32_t n_tok,
+                               int32_t np_grid, int32_t k, const float* logits, const float* head_stats,
+                               const int32_t* cur_pos, int32_t* kept_idx, void* workspace, size_t workspace_bytes,
+                               cudaStream_t stream) {
+  if (!ctx || !logits || !head_stats || !kept_idx || batch < 1 || heads < 1 || n_global < 1) return SPV_ERR_INVALID_ARG;
+  const int n_cur = n_tok - n_global;
+  if (n_cur < 1 || n_cur > np_grid || k < 1 || k > n_cur) return SPV_ERR_INVALID_ARG;
+  const int npad = (int)spv_align_up((size_t)np_grid, 4);
+  const size_t half = spv_align_up((size_t)batch * npad * sizeof(float), 256);
+  if (!workspace || workspace_bytes < 2 * half || ((uintptr_t)workspace & 255u)) return SPV_ERR_WORKSPACE;
+  float* mean_ws = (float*)workspace;
+  uint32_t* key_ws = (uint32_t*)((char*)workspace + half);
+  SpvProfScope prof(ctx, SPV_K_FILTER_SELECT, stream,
+                    (double)batch * ((double)heads * n_cur * 4.0 + (double)k * 4.0));
+  // key 0 ranks below every real key: padding and positions that are no longer present
+  SPV_CUDA_OK(cudaMemsetAsync(key_ws, 0, (size_t)batch * npad * sizeof(uint32_t), stream));
+  filter_mean_key_logits<<<dim3((n_cur + 255) / 256, batch), 256, 0, stream>>>(logits, head_stats, heads, n_global,
+                                                                             n_tok, cur_pos, npad, mean_ws, key_ws);
+  filter_select<<<batch, kSelThreads, 0, stream>>>(key_ws, np_grid, npad, k, kept_idx, nullptr, nullptr);
+  return spv_launch_ok(ctx, 2);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -177,14 +177,14 @@ __global__ void __launch_bounds__(32) mb_tma_kernel(const __grid_constant__ CUte
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tm);
-    uint32_t tile = (uint32_t)blockIdx.x * 7919u;
+    uint32_t tile = ((uint32_t)blockIdx.x * 7919u) & (uint32_t)(a.n_tiles - 1);
     const long long t0 = clock64();
 #pragma unroll 1
     for (int i = 0; i < a.iters; ++i) {
       const int s = i % a.stages;
       if (i >= a.stages) mbar_wait(&bars[s], ((i / a.stages) - 1) & 1, abort_flag, a.status, 0x3200);
       mbar_expect_tx(&bars[s], (uint32_t)box_bytes);
-      tile = (tile + 104729u) % (uint32_t)a.n_tiles;
+      tile = (tile + 104729u) & (uint32_t)(a.n_tiles - 1);          // n_tiles is a power of two
       tma_load_2d(smem + s * box_bytes, &tm, &bars[s], 0, (int)tile * a.box_rows);
     }
     // drain: every stage's last load
@@ -262,7 +262,8 @@ extern "C" int32_t spv_microbench(spv_ctx* ctx, const spv_microbench_desc* d, vo
         if (smem > 200 * 1024) { st = SPV_ERR_INVALID_ARG; break; }
         // the buffer the loads walk over: at most 32 MB, so that it stays in L2
         size_t span = rest_bytes > ((size_t)32 << 20) ? ((size_t)32 << 20) : rest_bytes;
-        const int n_tiles = (int)(span / (size_t)box_bytes);
+        int n_tiles = 1;
+        while ((size_t)(2 * n_tiles) * (size_t)box_bytes <= span) n_tiles *= 2;    // a power of two of tiles
         if (n_tiles < 64) { st = SPV_ERR_WORKSPACE; break; }
         CUtensorMap tm;
         const uint64_t dims[2] = {64, (uint64_t)n_tiles * d->box_rows};

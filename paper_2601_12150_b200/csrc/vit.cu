@@ -195,7 +195,7 @@ struct VitLayout {
   // filter stages: block after which each runs, tokens it keeps, entries per image over all stages
   int32_t n_stage, st_layer[SPV_MAX_FILTERS], st_k[SPV_MAX_FILTERS], k_total;
   size_t x0, x1, h, qkv, o, h1, h3, im2col, w_pe_pad, pos_bm, scores, mask, mark, mark2, rank, bm_pos, bm_of_pos, pos2,
-      pos3, kept_bm, kept_rm, out_row, plan, plan_bytes, glob, glob_bytes, filt, filt_bytes, total;
+      pos3, kept_bm, kept_rm, out_row, head_stats, plan, plan_bytes, glob, glob_bytes, filt, filt_bytes, total;
 };
 
 int32_t vit_layout(const spv_vit_config* c, int32_t batch, int32_t gh, int32_t gw, VitLayout* L) {
@@ -256,7 +256,8 @@ int32_t vit_layout(const spv_vit_config* c, int32_t batch, int32_t gh, int32_t g
   L->h3 = take(c->mlp_kind == SPV_MLP_SWIGLU ? rows * HID * 2 : 0);
   L->w_pe_pad = take((size_t)D * L->kpad * 2);
   L->pos_bm = take((size_t)L->np0 * D * 4);
-  L->scores = take((size_t)batch * c->heads * L->np0 * 4);
+  L->scores = take(c->unfused_filter ? (size_t)batch * c->heads * L->np0 * 4 : 0);
+  L->head_stats = take((size_t)batch * c->heads * 2 * 4);
   L->mask = take((size_t)batch * L->np0 * 4);
   L->mark = take((size_t)batch * L->np0 * 4);
   L->mark2 = take(L->n_stage > 1 ? (size_t)batch * L->np0 * 4 : 0);
@@ -324,6 +325,8 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
   __nv_bfloat16* w_pe_pad = (__nv_bfloat16*)(ws + L.w_pe_pad);
   float* pos_bm = (float*)(ws + L.pos_bm);
   float* scores = (float*)(ws + L.scores);
+  float* head_stats = (float*)(ws + L.head_stats);
+  const float* cls_logits = nullptr;
   float* mask = (float*)(ws + L.mask);
   float* mark = (float*)(ws + L.mark);
   float* mark2 = (float*)(ws + L.mark2);
@@ -407,12 +410,20 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
       // CLS->patch scores land at the tokens' ORIGINAL positions, so that the ranking breaks
       // ties by the lower original index
       const bool want_scores = stage < L.n_stage && l == L.st_layer[stage] && !forced_keep;
-      // a later stage ranks over the whole grid: positions that are gone hold NaN, which ranks last
-      if (want_scores && stage > 0)
-        SPV_CUDA_OK(cudaMemsetAsync(scores, 0xFF, (size_t)batch * H * np0 * 4, stream));
-      if ((st = spv_attn_run_globals(ctx, &plan, &io, want_scores ? scores : nullptr, want_scores ? cur_pos : nullptr,
-                                     np0, ws + L.glob, L.glob_bytes, stream)) != SPV_OK)
-        return st;
+      if (want_scores && !c->unfused_filter) {
+        // fused: the global kernels leave the logits and per-head (maximum, 1 / sum); the filter's first kernel
+        // evaluates the weights itself, so the [batch, heads, patches] score tensor is never written
+        if ((st = spv_attn_run_globals(ctx, &plan, &io, nullptr, nullptr, np0, ws + L.glob, L.glob_bytes, stream,
+                                       head_stats, &cls_logits)) != SPV_OK)
+          return st;
+      } else {
+        // a later stage ranks over the whole grid: positions that are gone hold NaN, which ranks last
+        if (want_scores && stage > 0)
+          SPV_CUDA_OK(cudaMemsetAsync(scores, 0xFF, (size_t)batch * H * np0 * 4, stream));
+        if ((st = spv_attn_run_globals(ctx, &plan, &io, want_scores ? scores : nullptr,
+                                       want_scores ? cur_pos : nullptr, np0, ws + L.glob, L.glob_bytes, stream)) != SPV_OK)
+          return st;
+      }
     }
     {
       spv_gemm_desc g{};
@@ -452,11 +463,17 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
         kept_stride = L.k_total;
       } else {
         // rank on the head-averaged scores in original-position order -> ascending original indices
-        spv_filter_desc fd{};
-        fd.batch = batch; fd.heads = H; fd.n_patch = np0; fd.n_global = G; fd.dim = 0; fd.keep_ratio = 1.0;
-        if ((st = spv_filter_run_k(ctx, &fd, k, scores, nullptr, nullptr, kept_rm, nullptr, nullptr, nullptr,
-                                   ws + L.filt, L.filt_bytes, stream)) != SPV_OK)
-          return st;
+        if (!c->unfused_filter) {
+          if ((st = spv_filter_rank_logits(ctx, batch, H, G, (int32_t)n, np0, k, cls_logits, head_stats, cur_pos,
+                                           kept_rm, ws + L.filt, L.filt_bytes, stream)) != SPV_OK)
+            return st;
+        } else {
+          spv_filter_desc fd{};
+          fd.batch = batch; fd.heads = H; fd.n_patch = np0; fd.n_global = G; fd.dim = 0; fd.keep_ratio = 1.0;
+          if ((st = spv_filter_run_k(ctx, &fd, k, scores, nullptr, nullptr, kept_rm, nullptr, nullptr, nullptr,
+                                     ws + L.filt, L.filt_bytes, stream)) != SPV_OK)
+            return st;
+        }
         kept_positions = kept_rm;
         kept_stride = k;
       }

@@ -179,6 +179,21 @@ def test_vit_forward_one_stage_list_equals_single_fields(ctx):
     assert np.array_equal(a, b) and np.array_equal(ka, kb)
 
 
+@pytest.mark.parametrize("stages,G", [([(1, 0.5)], 1), ([(1, 0.7), (2, 0.45)], 2)])
+def test_fused_filter_front_end_is_bit_identical(ctx, stages, G):
+    """The filter's fused front end (softmax weights of the CLS row, head mean and ranking keys in one kernel,
+    no [batch, heads, patches] score tensor) keeps exactly the tokens the two separate kernels keep."""
+    arch = synth.vit_tiny(layers=3, dim=128, heads=2, hidden=256, patch=4, n_global=G)
+    gh, gw = 21, 19
+    w = synth.vit_weights(8, arch, gh, gw, pos_base=4)
+    image = synth.tissue_batch(9, 3, gh * 4, gw * 4)
+    cfg = dict(arch, attn_mode=synth.ATTN_SPARSE, block=4, radius=1, filters=stages)
+    a, ka = _gpu_forward(ctx, cfg, w, image, gh, gw)
+    b, kb = _gpu_forward(ctx, dict(cfg, unfused_filter=1), w, image, gh, gw)
+    assert np.array_equal(ka, kb)
+    assert np.array_equal(a, b)
+
+
 @pytest.mark.parametrize("G", [5, 9, 16])
 def test_vit_forward_register_tokens(ctx, G):
     """CLS plus register tokens as global tokens (all attend everything and are attended by everything; the
