@@ -114,10 +114,12 @@ def forward_flops(wl, kept_positions):
     return dict(gemm=gemm, attn_patch=attn_patch, attn_global=attn_glob)
 
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per GEMM launch, averaged over the 104
-# GEMM launches of one step, from one ncu capture (profiles/gemm_dram_vitl16_2048_b4.md).  Valid
-# only for the kernel source it was taken with: reported as null once gemm.cu has changed.
-GEMM_TRAFFIC = {"vitl16_2048_b4_sparse_filter": (375.5e6, "39d36c0b6203")}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per GEMM launch, averaged over the 100 GEMM
+# launches of one step: four ncu captures, one per GEMM shape of a block at M = 65540 (two launches each),
+# weighted by the step's launch counts, the half-size launches after the filter scaled by their rows
+# (profiles/gemm_dram_by_shape_m65540.md).  Valid only for the kernel source it was taken with: reported as
+# null once gemm.cu has changed.
+GEMM_TRAFFIC = {"vitl16_2048_b4_sparse_filter": (393.6e6, "3ed141e24586")}
 
 
 def gemm_traffic(workload):

@@ -48,7 +48,9 @@ enum {
 typedef struct spv_ctx spv_ctx; /* device id, device status word, cached driver entry points */
 
 /* Create / destroy a context for CUDA device `device` (host calls; create allocates a few
- * bytes of device memory for the status word). */
+ * bytes of device memory for the status words).  A context belongs to that device: every entry
+ * point that takes it returns SPV_ERR_INVALID_ARG when another device is current on the calling
+ * thread.  One context per device and per host thread that issues calls. */
 int32_t spv_create(spv_ctx** out, int32_t device);
 int32_t spv_destroy(spv_ctx* ctx);
 /* Static description of a status code (host string, never NULL). */

@@ -654,12 +654,16 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 // ------------------------------------------------------------------------------------------
 constexpr int GCH = 128;   // fewest keys per CTA (bounds the number of chunk partials)
 
-// grid (heads, chunks, batch * G).  One pass over the chunk's keys: every group of eight lanes walks
-// keys k0 + grp, k0 + grp + 32, ... with its own running (max, sum, sum p*v) -- the key and the value
-// row of a key are loaded together, so twice as many loads are in flight as with a score pass
-// followed by a value pass -- and the 32 group states are merged through shared memory.  Writes the
-// chunk's (max, sum, sum p*v) and, when the scores are wanted, the scaled logits.
-template <bool kLogits>
+// grid (heads, chunks, batch * ceil(G / GQ)).  One pass over the chunk's keys serves GQ global queries (GQ = 1 is
+// what runs: with four queries per pass K and V cross HBM once per four queries, but the eight-lane dot products
+// and their shuffles then make the kernel instruction-bound -- 3.5 ms instead of 4.0 per step for five global
+// tokens, 5.8 instead of 4.5 for nine; the later queries' passes find K and V in L2 anyway): every group of
+// eight lanes walks keys k0 + grp, k0 + grp + 32, ...
+// with its own running (max, sum, sum p*v) per query -- the key and the value row of a key are loaded together,
+// so twice as many loads are in flight as with a score pass followed by a value pass -- and the 32 group states
+// are merged through shared memory, query after query.  Writes the chunk's (max, sum, sum p*v) of every query
+// and, when the scores are wanted, the scaled logits of global token 0.
+template <bool kLogits, int GQ>
 __global__ void __launch_bounds__(256, 2) attn_global_partial(const __nv_bfloat16* __restrict__ q,
                                                            const __nv_bfloat16* __restrict__ k,
                                                            const __nv_bfloat16* __restrict__ v, int64_t sb,
@@ -670,20 +674,29 @@ __global__ void __launch_bounds__(256, 2) attn_global_partial(const __nv_bfloat1
   __shared__ float s_m[32], s_l[32];
   __shared__ float s_o[32][HD + 1];
   // heads fastest: the CTAs running together read whole token rows (all heads) of one key chunk
-  const int h = blockIdx.x, chunk = blockIdx.y, bg = blockIdx.z;
-  const int b = bg / n_global, g = bg % n_global;
+  const int h = blockIdx.x, chunk = blockIdx.y;
+  const int g_chunks = (n_global + GQ - 1) / GQ;
+  const int b = blockIdx.z / g_chunks, g0 = (blockIdx.z % g_chunks) * GQ;
   const int k0 = chunk * chunk_len, k1 = min(k0 + chunk_len, n_tok);
   const int sub = threadIdx.x & 7, grp = threadIdx.x >> 3;   // 8 lanes per key, 32 keys in flight
-  float qf[8];
-  unpack8(__ldg(reinterpret_cast<const uint4*>(q + b * sb + (int64_t)g * st + (int64_t)h * sh) + sub), qf);
-  float* lg = logits + ((size_t)bg * heads + h) * n_tok;
-  float m = -INFINITY, l = 0.f;
-  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  float qf[GQ][8];
+#pragma unroll
+  for (int gq = 0; gq < GQ; ++gq) {
+    const int g = min(g0 + gq, n_global - 1);                // past the last query: a copy of it, never written
+    unpack8(__ldg(reinterpret_cast<const uint4*>(q + b * sb + (int64_t)g * st + (int64_t)h * sh) + sub), qf[gq]);
+  }
+  float* lg = logits + ((size_t)(b * n_global) * heads + h) * n_tok;     // row of global token 0
+  float m[GQ], l[GQ], acc[GQ][8];
+#pragma unroll
+  for (int gq = 0; gq < GQ; ++gq) {
+    m[gq] = -INFINITY; l[gq] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[gq][i] = 0.f;
+  }
   // the trip count is the same for every lane (the shuffles name the whole warp); keys past the
-  // end of the chunk are predicated off.  The loads of GU keys (key and value rows) are issued
-  // before any of them is used.
-  constexpr int GU = 4;
-  // the loads of the next GU keys are in flight while the current ones are used
+  // end of the chunk are predicated off.  The loads of the next GU keys (key and value rows) are in flight
+  // while the current ones are used.
+  constexpr int GU = GQ == 1 ? 4 : 2;
   auto load_batch = [&](int kk0, uint4* ku, uint4* vu) {
 #pragma unroll
     for (int u = 0; u < GU; ++u) {
@@ -705,73 +718,80 @@ __global__ void __launch_bounds__(256, 2) attn_global_partial(const __nv_bfloat1
 #pragma unroll
     for (int u = 0; u < GU; ++u) { ku[u] = kn[u]; vu[u] = vn[u]; }
     if (kk0 + 32 * GU < k1) load_batch(kk0 + 32 * GU, kn, vn);
-    float d[GU];
+    float kf[GU][8], vf[GU][8];
 #pragma unroll
-    for (int u = 0; u < GU; ++u) {
-      float kf[8];
-      unpack8(ku[u], kf);
-      d[u] = 0.f;
+    for (int u = 0; u < GU; ++u) { unpack8(ku[u], kf[u]); unpack8(vu[u], vf[u]); }
 #pragma unroll
-      for (int i = 0; i < 8; ++i) d[u] = fmaf(qf[i], kf[i], d[u]);
-    }
+    for (int gq = 0; gq < GQ; ++gq) {
+      float d[GU];
 #pragma unroll
-    for (int u = 0; u < GU; ++u) {
-      d[u] += __shfl_xor_sync(0xffffffffu, d[u], 1);
-      d[u] += __shfl_xor_sync(0xffffffffu, d[u], 2);
-      d[u] += __shfl_xor_sync(0xffffffffu, d[u], 4);
-      d[u] = (kk0 + u * 32 + grp < k1) ? d[u] * scale : -INFINITY;
-    }
-    if (kLogits && sub < GU) {
-      // lane u of the group writes key u's logit
-      float mine = d[0];
+      for (int u = 0; u < GU; ++u) {
+        d[u] = 0.f;
 #pragma unroll
-      for (int u = 1; u < GU; ++u) mine = sub == u ? d[u] : mine;
-      const int kk = kk0 + sub * 32 + grp;
-      if (kk < k1) lg[kk] = mine;
-    }
-    float mx = d[0];
+        for (int i = 0; i < 8; ++i) d[u] = fmaf(qf[gq][i], kf[u][i], d[u]);
+      }
 #pragma unroll
-    for (int u = 1; u < GU; ++u) mx = fmaxf(mx, d[u]);
-    if (mx > m) {                        // the same decision in all eight lanes of the group
-      const float a = __expf(m - mx);    // m = -inf on the first batch: a = 0, the state is empty
-      l *= a;
+      for (int u = 0; u < GU; ++u) {
+        d[u] += __shfl_xor_sync(0xffffffffu, d[u], 1);
+        d[u] += __shfl_xor_sync(0xffffffffu, d[u], 2);
+        d[u] += __shfl_xor_sync(0xffffffffu, d[u], 4);
+        d[u] = (kk0 + u * 32 + grp < k1) ? d[u] * scale : -INFINITY;
+      }
+      if (kLogits && g0 + gq == 0 && sub < GU) {
+        // lane u of the group writes key u's logit
+        float mine = d[0];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] *= a;
-      m = mx;
-    }
-    const float mref = m == -INFINITY ? 0.f : m;   // a group that has seen no key yet: every p below is 0
+        for (int u = 1; u < GU; ++u) mine = sub == u ? d[u] : mine;
+        const int kk = kk0 + sub * 32 + grp;
+        if (kk < k1) lg[kk] = mine;
+      }
+      float mx = d[0];
 #pragma unroll
-    for (int u = 0; u < GU; ++u) {
-      const float pw = __expf(d[u] - mref);          // 0 for a key past the end of the chunk
-      float vf[8];
-      unpack8(vu[u], vf);
-      l += pw;
+      for (int u = 1; u < GU; ++u) mx = fmaxf(mx, d[u]);
+      if (mx > m[gq]) {                      // the same decision in all eight lanes of the group
+        const float a = __expf(m[gq] - mx);  // m = -inf on the first batch: a = 0, the state is empty
+        l[gq] *= a;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] = fmaf(pw, vf[i], acc[i]);
+        for (int i = 0; i < 8; ++i) acc[gq][i] *= a;
+        m[gq] = mx;
+      }
+      const float mref = m[gq] == -INFINITY ? 0.f : m[gq];   // a group that has seen no key yet: every p below is 0
+#pragma unroll
+      for (int u = 0; u < GU; ++u) {
+        const float pw = __expf(d[u] - mref);          // 0 for a key past the end of the chunk
+        l[gq] += pw;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[gq][i] = fmaf(pw, vf[u][i], acc[gq][i]);
+      }
     }
   }
-  if (sub == 0) { s_m[grp] = m; s_l[grp] = l; }
 #pragma unroll
-  for (int i = 0; i < 8; ++i) s_o[grp][sub * 8 + i] = acc[i];
-  __syncthreads();
-  float cmax = -INFINITY;
+  for (int gq = 0; gq < GQ; ++gq) {
+    if (g0 + gq >= n_global) break;                          // uniform over the CTA
+    if (gq > 0) __syncthreads();                             // the previous query's merge has read the arrays
+    if (sub == 0) { s_m[grp] = m[gq]; s_l[grp] = l[gq]; }
 #pragma unroll
-  for (int gI = 0; gI < 32; ++gI) cmax = fmaxf(cmax, s_m[gI]);
-  const size_t pidx = ((size_t)bg * heads + h) * n_chunks + chunk;
-  if (threadIdx.x < HD) {
-    float t = 0.f;
+    for (int i = 0; i < 8; ++i) s_o[grp][sub * 8 + i] = acc[gq][i];
+    __syncthreads();
+    float cmax = -INFINITY;
 #pragma unroll
-    for (int gI = 0; gI < 32; ++gI)
-      if (s_m[gI] > -INFINITY) t += s_o[gI][threadIdx.x] * __expf(s_m[gI] - cmax);
-    part_o[pidx * HD + threadIdx.x] = t;
-  }
-  if (threadIdx.x == 0) {
-    float t = 0.f;
+    for (int gI = 0; gI < 32; ++gI) cmax = fmaxf(cmax, s_m[gI]);
+    const size_t pidx = ((size_t)(b * n_global + g0 + gq) * heads + h) * n_chunks + chunk;
+    if (threadIdx.x < HD) {
+      float t = 0.f;
 #pragma unroll
-    for (int gI = 0; gI < 32; ++gI)
-      if (s_m[gI] > -INFINITY) t += s_l[gI] * __expf(s_m[gI] - cmax);
-    part_ml[pidx * 2] = cmax;
-    part_ml[pidx * 2 + 1] = t;
+      for (int gI = 0; gI < 32; ++gI)
+        if (s_m[gI] > -INFINITY) t += s_o[gI][threadIdx.x] * __expf(s_m[gI] - cmax);
+      part_o[pidx * HD + threadIdx.x] = t;
+    }
+    if (threadIdx.x == 0) {
+      float t = 0.f;
+#pragma unroll
+      for (int gI = 0; gI < 32; ++gI)
+        if (s_m[gI] > -INFINITY) t += s_l[gI] * __expf(s_m[gI] - cmax);
+      part_ml[pidx * 2] = cmax;
+      part_ml[pidx * 2 + 1] = t;
+    }
   }
 }
 
@@ -963,7 +983,8 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   const size_t rows = (size_t)B * G * io->heads;
   // as many chunks as fill the GPU once (two CTAs of this kernel per SM), none shorter than GCH keys
   const int max_chunks = (n_tok + GCH - 1) / GCH;
-  int chunks = (int)((size_t)ctx->sm_count * 2 / rows);
+  const size_t ctas_per_chunk = (size_t)B * G * io->heads;
+  int chunks = (int)((size_t)ctx->sm_count * 2 / ctas_per_chunk);
   chunks = chunks < 1 ? 1 : (chunks > max_chunks ? max_chunks : chunks);
   const int chunk_len = ((n_tok + chunks - 1) / chunks + 127) / 128 * 128;
   chunks = (n_tok + chunk_len - 1) / chunk_len;
@@ -973,12 +994,13 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   float* part_o = (float*)w;
   SpvProfScope prof(ctx, SPV_K_ATTN_GLOBAL, stream);
   if (logits_out) *logits_out = logits;
-  if (scores || head_stats) attn_global_partial<true><<<dim3(io->heads, chunks, B * G), 256, 0, stream>>>(
-      (const __nv_bfloat16*)io->q, (const __nv_bfloat16*)io->k, (const __nv_bfloat16*)io->v, io->sb, io->st, io->sh,
-      n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks, chunk_len);
-  else attn_global_partial<false><<<dim3(io->heads, chunks, B * G), 256, 0, stream>>>(
-      (const __nv_bfloat16*)io->q, (const __nv_bfloat16*)io->k, (const __nv_bfloat16*)io->v, io->sb, io->st, io->sh,
-      n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks, chunk_len);
+  const bool lg_on = scores || head_stats;
+#define SPV_GLOBAL_PARTIAL(LG, GQ_)                                                                                  \
+  attn_global_partial<LG, GQ_><<<dim3(io->heads, chunks, B * ((G + GQ_ - 1) / GQ_)), 256, 0, stream>>>(              \
+      (const __nv_bfloat16*)io->q, (const __nv_bfloat16*)io->k, (const __nv_bfloat16*)io->v, io->sb, io->st, io->sh, \
+      n_tok, G, io->heads, io->scale, logits, part_ml, part_o, chunks, chunk_len)
+  if (lg_on) SPV_GLOBAL_PARTIAL(true, 1); else SPV_GLOBAL_PARTIAL(false, 1);
+#undef SPV_GLOBAL_PARTIAL
   attn_global_combine<<<dim3(io->heads, B * G), 256, 0, stream>>>(logits, part_ml, part_o, chunks, n_tok, G,
                                                                  io->heads, (__nv_bfloat16*)io->o, io->o_sb,
                                                                  io->o_st, io->o_sh, scores, score_idx, score_stride,
@@ -1023,6 +1045,7 @@ extern "C" int32_t spatial_block_attention(spv_ctx* ctx, const spv_attn_desc* d,
                                            size_t workspace_bytes, void* stream_) {
   if (!ctx) return SPV_ERR_INVALID_ARG;
   int32_t st = validate_desc(d);
+  if (spv_on_device(ctx) != SPV_OK) return SPV_ERR_INVALID_ARG;
   if (st != SPV_OK) return st;
   if (!q || !k || !v || !o) return SPV_ERR_INVALID_ARG;
   if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15u) return SPV_ERR_ALIGNMENT;

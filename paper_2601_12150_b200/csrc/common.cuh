@@ -29,7 +29,6 @@ struct spv_ctx {
   int32_t prof_on;
   // one-time per-device launch configuration (function attributes are per device, and a context is bound to one)
   int32_t attn_configured;
-  int32_t attn_ctas_per_sm[2];   // resident CTAs of the attention kernel per SM: up to 8 / up to 16 global tokens
   int32_t gemm_single_configured[8];   // per epilogue variant
   int32_t gemm_max_pairs[8];     // per epilogue variant: CTA pairs of the pair-form GEMM that can be resident at
                                  // once (0 = not yet queried)
@@ -56,6 +55,14 @@ struct SpvProfScope {
     cudaError_t _e = (expr);                      \
     if (_e != cudaSuccess) return SPV_ERR_CUDA;   \
   } while (0)
+
+// A context belongs to one device (its status words, function attributes and SM count are that device's): the
+// entry points refuse to run when another device is current on the calling thread.
+static inline int32_t spv_on_device(const spv_ctx* ctx) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SPV_ERR_CUDA;
+  return dev == ctx->device ? SPV_OK : SPV_ERR_INVALID_ARG;
+}
 
 static inline int32_t spv_launch_ok(spv_ctx* ctx, int n = 1) {
   ctx->launches += n;

@@ -148,6 +148,7 @@ __global__ void selftest_wait_kernel(uint32_t limit_ns, uint32_t* status) {
 
 extern "C" int32_t spv_selftest_wait(spv_ctx* ctx, uint32_t limit_ns, void* stream) {
   if (!ctx) return SPV_ERR_INVALID_ARG;
+  if (spv_on_device(ctx) != SPV_OK) return SPV_ERR_INVALID_ARG;
   if (limit_ns > 1000000u) limit_ns = 1000000u;
   selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_ns, ctx->d_status);
   return spv_launch_ok(ctx);

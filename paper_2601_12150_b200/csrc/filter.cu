@@ -261,6 +261,7 @@ int32_t spv_filter_run_k(spv_ctx* ctx, const spv_filter_desc* d, int32_t k, cons
                          const int32_t* pos_in, int32_t* pos_out, void* workspace, size_t workspace_bytes,
                          cudaStream_t stream) {
   if (!ctx || !d || k < 1 || k > d->n_patch) return SPV_ERR_INVALID_ARG;
+  if (spv_on_device(ctx) != SPV_OK) return SPV_ERR_INVALID_ARG;
   if (!scores || !kept_idx) return SPV_ERR_INVALID_ARG;
   if ((tokens_in == nullptr) != (tokens_out == nullptr)) return SPV_ERR_INVALID_ARG;
   if (tokens_in && d->dim == 0) return SPV_ERR_INVALID_ARG;

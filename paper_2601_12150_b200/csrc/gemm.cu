@@ -426,6 +426,7 @@ int32_t launch(spv_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tw, const
 extern "C" int32_t spv_gemm_bf16(spv_ctx* ctx, const spv_gemm_desc* d, const void* a, const void* w, void* out,
                                  void* stream_) {
   if (!ctx || !d || !a || !w || !out) return SPV_ERR_INVALID_ARG;
+  if (spv_on_device(ctx) != SPV_OK) return SPV_ERR_INVALID_ARG;
   if (d->m < 1 || d->n < 1 || d->k < 1) return SPV_ERR_INVALID_ARG;
   if (d->k % 8 || d->n % 8 || d->lda % 8 || d->ldw % 8 || d->ldo % 8) return SPV_ERR_ALIGNMENT;
   if (d->lda < d->k || d->ldw < d->k || d->ldo < d->n) return SPV_ERR_INVALID_ARG;

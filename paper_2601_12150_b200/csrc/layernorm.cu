@@ -106,6 +106,7 @@ __global__ void __launch_bounds__(256, (kMaxVec <= 8 ? 2 : 1)) layernorm_kernel(
 extern "C" int32_t spv_layernorm(spv_ctx* ctx, const float* x, int64_t rows, int32_t dim, const float* gamma,
                                  const float* beta, float eps, void* y, const int32_t* out_row, void* stream) {
   if (!ctx || !x || !gamma || !beta || !y || rows < 1 || dim < 8) return SPV_ERR_INVALID_ARG;
+  if (spv_on_device(ctx) != SPV_OK) return SPV_ERR_INVALID_ARG;
   if (dim % 8) return SPV_ERR_ALIGNMENT;
   if (((uintptr_t)x & 15u) || ((uintptr_t)y & 15u) || ((uintptr_t)gamma & 15u) || ((uintptr_t)beta & 15u))
     return SPV_ERR_ALIGNMENT;

@@ -201,6 +201,7 @@ __global__ void __launch_bounds__(32) mb_tma_kernel(const __grid_constant__ CUte
 extern "C" int32_t spv_microbench(spv_ctx* ctx, const spv_microbench_desc* d, void* buffer, size_t buffer_bytes,
                                   void* stream_, spv_microbench_result* out) {
   if (!ctx || !d || !out || !buffer) return SPV_ERR_INVALID_ARG;
+  if (spv_on_device(ctx) != SPV_OK) return SPV_ERR_INVALID_ARG;
   if (d->iters < 1 || d->iters > (1 << 22) || d->ctas_per_sm < 1 || d->ctas_per_sm > 4) return SPV_ERR_INVALID_ARG;
   if ((uintptr_t)buffer & 255u) return SPV_ERR_WORKSPACE;
   cudaStream_t stream = (cudaStream_t)stream_;

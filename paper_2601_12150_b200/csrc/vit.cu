@@ -303,6 +303,7 @@ extern "C" int32_t vit_forward(spv_ctx* ctx, const spv_vit_config* c, const spv_
                                int32_t batch, int32_t gh, int32_t gw, void* out_tokens, int32_t* kept_idx,
                                const int32_t* forced_keep, void* workspace, size_t workspace_bytes, void* stream_) {
   if (!ctx || !w || !image || !out_tokens || !w->layer) return SPV_ERR_INVALID_ARG;
+  if (spv_on_device(ctx) != SPV_OK) return SPV_ERR_INVALID_ARG;
   VitLayout L;
   int32_t st = vit_layout(c, batch, gh, gw, &L);
   if (st != SPV_OK) return st;

@@ -46,7 +46,8 @@ def _check_scores(got, ref):
 
 def _check_topk_of_mean(got, ref, keep=0.5):
     """The kept set of Sec. 3.3 from the GPU's scores equals the one from the oracle's scores, apart from
-    tokens whose oracle mean lies within 1e-3 relative of the oracle's threshold."""
+    tokens whose oracle mean lies within 1e-3 relative of the oracle's threshold (here both sides start from
+    the same bf16 Q and K, so only the accumulation order differs)."""
     for b in range(ref.shape[0]):
         mg, mw = got[b].astype(np.float64).mean(axis=0), ref[b].astype(np.float64).mean(axis=0)
         k = int(np.ceil(keep * mw.size - 1e-9))

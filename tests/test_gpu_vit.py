@@ -4,8 +4,15 @@ the token filter of Sec. 3.3) against the CPU oracle on the same seeded weights 
 Tolerance for the bf16 output tokens vs the oracle: max |err| <= 2e-2 and relative L2 <= 5e-3.
 The filter decides an integer result from scores that the two sides compute in different
 precisions, so the comparison runs twice: free-running (kept sets may differ only in tokens whose
-oracle score sits within 1e-3 relative of the oracle's threshold score) and teacher-forced (the
-oracle is re-run with the GPU's kept indices, then the tensor tolerances apply)."""
+oracle score sits within THRESHOLD_REL of the oracle's threshold score) and teacher-forced (the
+oracle is re-run with the GPU's kept indices, then the tensor tolerances apply).
+
+THRESHOLD_REL = 2^-8: the GPU forms the CLS logits from bf16 q and k, i.e. from operands that carry a
+relative rounding error of up to half a bf16 ulp, 2^-8; a softmax weight inherits the logit's absolute
+error as a relative one.  With trained-looking (peaked) score rows few tokens sit that close to the
+threshold; with the nearly uniform rows random weights give on a 146x146 grid (every weight within a few
+1e-4 relative of 1/N) the ranking near the threshold is decided below the operands' precision, and the
+bound says exactly how far a disagreeing token may be from it."""
 import numpy as np
 import pytest
 import torch
@@ -22,6 +29,9 @@ def ctx():
     c = spv.Context(0)
     yield c
     c.close()
+
+
+THRESHOLD_REL = 2.0 ** -8
 
 
 def _check(got, ref, max_abs=2e-2, rel_l2=5e-3):
@@ -127,10 +137,15 @@ def _compare(ctx, arch, cfg, gh, gw, B, seed, w=None, image=None, report=None, f
                 first.pop("filters")
                 first["filter_layer"], first["keep_ratio"] = full["filters"][0]
             mean = _mean_scores_of_oracle(first, w, image, gh, gw)
+            worst = 0.0
             for b in range(B):
                 thr = np.sort(mean[b])[::-1][k1 - 1]
                 diff = np.setxor1d(kept[b, :k1], okept[b, :k1])
-                assert (np.abs(mean[b][diff] - thr) <= 1e-3 * abs(thr)).all(), (b, diff, mean[b][diff], thr)
+                if diff.size:
+                    worst = max(worst, float((np.abs(mean[b][diff] - thr) / abs(thr)).max()))
+            if report is not None:
+                report["max_rel_distance_to_threshold_of_differing_tokens"] = worst
+            assert worst <= THRESHOLD_REL, worst
         ref = oracle.vit_forward(full, w, image, gh, gw, forced_keep=kept)
     fill_report(ref["out"])
     _check(got, ref["out"])

@@ -43,3 +43,17 @@ def test_host_only_entry_points():
     assert need.value >= 2 * 2 * 4096 * 4
     d.dim = 1001
     assert spv.lib().spv_filter_workspace_size(ctypes.byref(d), ctypes.byref(need)) == spv.ERR_ALIGNMENT
+
+
+def test_no_per_process_launch_state_in_the_kernels_sources():
+    """Launch configuration (function attributes, resident-CTA counts) is per device and lives in the context:
+    no function-level `static` variable may hold it in the CUDA sources (two contexts on two devices of one
+    process would share it)."""
+    import re
+    csrc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_2601_12150_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if not name.endswith(".cu"):
+            continue
+        text = open(os.path.join(csrc, name)).read()
+        for m in re.finditer(r"^\s+static\s+(bool|int|int32_t|unsigned)\s+\w+\s*(=|;)", text, re.M):
+            raise AssertionError(f"{name}: function-level static `{m.group(0).strip()}`")
