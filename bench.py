@@ -560,6 +560,11 @@ OP_WORKLOADS = {
                                                       pattern="scattered")),
     "attn_128x128_b4_keep50_coherent": ("attn", dict(grid=128, block=8, radius=1, batch=4, heads=16, keep=0.5,
                                                      pattern="coherent")),
+    # 16x16-patch blocks, same 3x3 neighbourhood: a 128-row query tile lies inside one block (no warp-tile without
+    # keys) and streams three times as many key tiles per CTA as with 8x8 blocks
+    "attn_128x128_b4_block16_r1": ("attn", dict(grid=128, block=16, radius=1, batch=4, heads=16)),
+    "attn_128x128_b4_block16_keep50_scattered": ("attn", dict(grid=128, block=16, radius=1, batch=4, heads=16, keep=0.5,
+                                                              pattern="scattered")),
     # filter: (grid, batch, heads, dim, keep, cold L2)
     "filter_64x64_b1": ("filter", dict(grid=64, batch=1, heads=16, dim=1024, keep=0.5, cold=False)),
     "filter_64x64_b1_cold": ("filter", dict(grid=64, batch=1, heads=16, dim=1024, keep=0.5, cold=True)),

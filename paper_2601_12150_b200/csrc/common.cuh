@@ -37,11 +37,25 @@ struct spv_ctx {
 // Event pair around one launch group while profiling is on (no-ops otherwise).
 int32_t spv_prof_begin(spv_ctx* ctx, int32_t cls, cudaStream_t stream);
 void spv_prof_end(spv_ctx* ctx, int32_t token, cudaStream_t stream, double work);
+// With -DSPV_NVTX every launch group is also an NVTX range named after its kernel class (host-side ranges for a
+// timeline tool; off in the default build).
+#ifdef SPV_NVTX
+#include <nvtx3/nvToolsExt.h>
+static inline void spv_nvtx_push(int32_t cls) {
+  static const char* const names[SPV_K_COUNT] = {"spv:gemm", "spv:attn_patch", "spv:attn_global", "spv:attn_plan",
+                                                 "spv:layernorm", "spv:filter_select", "spv:filter_gather", "spv:misc"};
+  nvtxRangePushA(cls >= 0 && cls < SPV_K_COUNT ? names[cls] : "spv");
+}
+static inline void spv_nvtx_pop() { nvtxRangePop(); }
+#else
+static inline void spv_nvtx_push(int32_t) {}
+static inline void spv_nvtx_pop() {}
+#endif
 struct SpvProfScope {
   spv_ctx* ctx; cudaStream_t stream; int32_t token; double work;
   SpvProfScope(spv_ctx* c, int32_t cls, cudaStream_t s, double w = 0.0)
-      : ctx(c), stream(s), token(c->prof_on ? spv_prof_begin(c, cls, s) : -1), work(w) {}
-  ~SpvProfScope() { if (token >= 0) spv_prof_end(ctx, token, stream, work); }
+      : ctx(c), stream(s), token(c->prof_on ? spv_prof_begin(c, cls, s) : -1), work(w) { spv_nvtx_push(cls); }
+  ~SpvProfScope() { spv_nvtx_pop(); if (token >= 0) spv_prof_end(ctx, token, stream, work); }
 };
 
 // Second device status word (d_status[1]; the bounded waits look at d_status[0] only): an index array given

@@ -20,13 +20,21 @@ def ctx():
     c.close()
 
 
+def _half_ulp_bf16(x):
+    """Half a unit in the last place of the bf16 number nearest to x (8 significand bits)."""
+    ax = np.maximum(np.abs(np.asarray(x, dtype=np.float64)), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(ax)) - 8)
+
+
 def _check(got, ref, max_abs=2e-2, rel_l2=5e-3):
-    """max |err| <= 2e-2 and relative L2 <= 5e-3; above |ref| = 2 the element bound is 1e-2 |ref| (half an ulp
-    of the bf16 output is up to 2^-8 |x|, which alone passes 2e-2 from |x| = 5.1 on)."""
-    err = got.astype(np.float64) - ref.astype(np.float64)
+    """max |err| <= 2e-2 and relative L2 <= 5e-3.  The outputs are stored as bf16: the 2e-2 is the budget of
+    the arithmetic (the value before it is rounded to the output format), and the rounding itself may add up
+    to half a bf16 ulp of the value, which alone passes 2e-2 from |x| = 4 on.  Element bound: 2e-2 + half_ulp."""
     assert np.isfinite(got).all()
-    bound = np.maximum(max_abs, 0.5 * max_abs * np.abs(ref.astype(np.float64)))
-    assert (np.abs(err) <= bound).all(), float((np.abs(err) / bound).max())
+    err = got.astype(np.float64) - ref.astype(np.float64)
+    bound = max_abs + _half_ulp_bf16(ref)
+    worst = np.unravel_index(np.argmax(np.abs(err) / bound), err.shape)
+    assert (np.abs(err) <= bound).all(), (worst, float(err[worst]), float(ref[worst]))
     rel = np.linalg.norm(err) / np.linalg.norm(ref)
     assert rel <= rel_l2, rel
 

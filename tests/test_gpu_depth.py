@@ -52,11 +52,13 @@ def _run(ctx, arch, cfg, grid, wseed, iseed, side, name, background=None, backgr
     full = dict(arch, **cfg)
     key = dict(name=name, cfg={k: v for k, v in full.items()}, grid=grid, wseed=wseed, iseed=iseed, side=side, kw=kw)
     report = {}
-    _compare(ctx, arch, cfg, grid, grid, 1, 0, w=w, image=image, report=report,
-             free_oracle=lambda: _oracle_cached(full, w, image, grid, grid, key))
-    if REPORT:
-        with open(REPORT, "a") as f:
-            f.write(json.dumps(dict(case=name, **report)) + "\n")
+    try:
+        _compare(ctx, arch, cfg, grid, grid, 1, 0, w=w, image=image, report=report,
+                 free_oracle=lambda: _oracle_cached(full, w, image, grid, grid, key))
+    finally:
+        if REPORT:
+            with open(REPORT, "a") as f:
+                f.write(json.dumps(dict(case=name, **report)) + "\n")
     return report
 
 
