@@ -3,7 +3,9 @@
 //
 // Three kernels on one stream:
 //   filter_mean_key   head average in fp32 (heads added in index order, one division) and an
-//                     order-preserving 32-bit key per patch;
+//                     order-preserving 32-bit key per patch; filter_mean_key_logits is the same with the
+//                     softmax weights evaluated on the fly from the global row's logits (the fused front end
+//                     inside vit_forward: the [batch, heads, patches] score tensor is never written);
 //   filter_select     one CTA per image: 4-pass radix select of the k-th largest key, then an
 //                     ordered two-counter scan that emits the kept indices in ascending order;
 //   filter_gather     128-bit row copy of the global tokens and the kept rows.

@@ -6,6 +6,9 @@
 // attention kernel then reads Q/K/V straight out of the QKV GEMM's output with no regrouping
 // copy in any layer, and the filter's stable compaction keeps the order block-major.  Only the
 // final LayerNorm scatters rows back to ascending original position, the exported order.
+// The filter may run after several blocks (up to SPV_MAX_FILTERS stages): every stage ranks over the whole
+// grid (positions that are gone rank last), marks the kept positions, compacts the residual stream and the
+// position list into the other of two buffers and rebuilds the attention plan from the new positions.
 //
 // The residual stream stays fp32 (LayerNorm reads it, the GEMM epilogues add into it); every
 // GEMM operand is bf16.

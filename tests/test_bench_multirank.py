@@ -54,3 +54,30 @@ def test_attention_pair_count_matches_golden_closed_forms():
     brute = int(((np.abs(by[:, None] - by[None]) <= 1) & (np.abs(bx[:, None] - bx[None]) <= 1)).sum())
     p, g = bench.attention_pairs(20, 12, 8, 1, 2, pos)
     assert p == brute + 90 * 2 and g == 2 * 92
+
+
+def test_kept_set_generators_and_config_line():
+    """The benchmark's kept-set generators (inputs of the coherent-set measurements) and the config object
+    shared by the two arms."""
+    import numpy as np
+    import bench
+    import synth
+    k = bench.coherent_kept(7, 64, 0.5)
+    assert k.dtype == np.int32 and k.size == 2048 and (np.diff(k) > 0).all() and k.min() >= 0 and k.max() < 4096
+    # coherent: far more allowed pairs than a scattered set of the same size
+    rng = np.random.default_rng(0)
+    sc = np.sort(rng.choice(4096, size=2048, replace=False))
+    assert bench.attention_pairs(64, 64, 8, 1, 1, k)[0] > 1.2 * bench.attention_pairs(64, 64, 8, 1, 1, sc)[0]
+    bm = bench.block_major(k, 64, 8)
+    blk = (bm // 64) // 8 * 8 + (bm % 64) // 8
+    assert (np.diff(blk) >= 0).all() and sorted(bm.tolist()) == k.tolist()
+    img = synth.tissue_batch(3, 2, 64, 64, background=0.5)
+    tk = bench.tissue_kept(img, 4, 100)
+    assert tk.shape == (2, 100) and (np.diff(tk, axis=1) > 0).all()
+    mean = img[:, 1].reshape(2, 16, 4, 16, 4).mean(axis=(2, 4)).reshape(2, 256)
+    for b in range(2):
+        assert mean[b][tk[b]].max() <= np.sort(mean[b])[100 - 1] + 1e-6          # the darkest 100
+    wl = bench.workload_config(bench.DEFAULT_WORKLOAD)
+    c = bench.config_of(wl, 1)
+    assert c["workload"] == bench.DEFAULT_WORKLOAD and c["kept"] == 8192 and c["tokens"] == 16385
+    assert bench.config_of(wl, 2)["parallelism"] == "replicas"
