@@ -31,17 +31,21 @@ constexpr int TQ = 128;            // query rows per tile (MMA M)
 constexpr int TK = 32;             // keys per tile (MMA N of S, K extent of P V): three S buffers of 32 columns and
                                    // O make 160 TMEM columns, so three CTAs fit an SM
 constexpr int HD = 64;             // head_dim
-constexpr int KST = 6;             // K / V smem stages (Q K^T runs up to two key tiles ahead of P V)
+// K / V shared-memory stages (Q K^T runs up to two key tiles ahead of P V; an even count, so that each of the
+// two Q K^T issuers always meets the same stages): six with up to 8 global tokens, four with 9-16, whose rows and
+// scores take 10 KB more -- three CTAs fit an SM either way.
+constexpr int kst_for(int grows) { return grows <= 8 ? 6 : 4; }
 constexpr int NSB = 3;             // S / P buffers in TMEM: a softmax warp may be two key tiles ahead of the slowest
 constexpr int ATT_THREADS = 256;   // warps 0-3 softmax (one warpgroup), 4 TMA, 5-7 MMA issue: the second warpgroup
                                    // hands most of its registers to the first
 constexpr int TILE_BYTES = 128 * 128;  // Q tile
 constexpr int KV_BYTES = TK * 128;      // K or V tile
 constexpr int MAXG = 16;           // global tokens
-// Shared memory of a CTA for `grows` rows of global tokens (8 or 16: with up to 8, three CTAs fit an SM):
+// Shared memory of a CTA for `grows` rows of global tokens (8 or 16):
 // Q tile, K / V stages, the global tokens' key and value rows (128 B each), barriers, their scores per query row.
 constexpr int att_smem(int grows) {
-  return TILE_BYTES + 2 * KST * KV_BYTES + 2 * grows * 128 + 1024 /*align*/ + 512 /*barriers*/ + grows * 128 * 4;
+  return TILE_BYTES + 2 * kst_for(grows) * KV_BYTES + 2 * grows * 128 + 1024 /*align*/ + 512 /*barriers*/ +
+         grows * 128 * 4;
 }
 // two TMEM allocations per CTA, 160 columns in all, so that three CTAs share an SM's 512: O and two S buffers in
 // the first, the third S buffer in the second.  A row's P (bf16, 16 columns) is written over its own S.
@@ -274,6 +278,7 @@ __device__ __forceinline__ void unpack8(const uint4& u, float* f) {
   }
 }
 
+template <int KST>
 __global__ void __launch_bounds__(ATT_THREADS, 3)
 attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kg,
@@ -938,7 +943,10 @@ int32_t spv_attn_plan_build(spv_ctx* ctx, int32_t batch, int32_t grid_h, int32_t
 
 int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, cudaStream_t stream) {
   if (!ctx->attn_configured) {
-    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, att_smem(MAXG)));
+    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel<kst_for(8)>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     att_smem(8)));
+    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel<kst_for(MAXG)>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     att_smem(MAXG)));
     ctx->attn_configured = 1;
   }
   const int n_tok = plan->n_global + plan->n_patch;
@@ -964,7 +972,10 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   // the output as a tensor map (same row order as Q, boxes of 32 rows): warps whose rows are all valid store by TMA
   CUtensorMap to;
   if ((st = make_qkv_map(ctx, &to, io->o, io->o_sb, io->o_st, io->o_sh, n_tok, io->heads, plan->batch, 32)) != SPV_OK) return st;
-  attn_patch_kernel<<<grid, ATT_THREADS, att_smem(pp.grows), stream>>>(tq, tk, tv, tkg, tvg, to, pp);
+  if (pp.grows == 8)
+    attn_patch_kernel<kst_for(8)><<<grid, ATT_THREADS, att_smem(8), stream>>>(tq, tk, tv, tkg, tvg, to, pp);
+  else
+    attn_patch_kernel<kst_for(MAXG)><<<grid, ATT_THREADS, att_smem(MAXG), stream>>>(tq, tk, tv, tkg, tvg, to, pp);
   return spv_launch_ok(ctx);
 }
 
