@@ -277,3 +277,30 @@ def test_random_geometries_both_token_orders(ctx, seed):
     _check(got_bm, reorder(want))
     for i in range(B):
         _check_scores(gsc_bm[i], wsc[i][:, perm[i]])
+
+
+def test_repeated_calls_are_bit_identical(ctx):
+    """The kernel's warps advance independently and its roles hand tiles over through barriers; whatever the
+    interleaving, the result may not change: the same call five times on a filtered, ragged geometry with nine
+    global tokens and on the 128x128 grid gives the same bits (a missed wait or a buffer reused too early would
+    show here first)."""
+    rng = np.random.default_rng(11)
+    for (gh, gw, b, r, G, B, H, keep) in [(37, 29, 8, 1, 9, 2, 3, 0.5), (128, 128, 8, 1, 1, 1, 4, None), (64, 64, 8, 2, 1, 2, 4, 0.4)]:
+        n0 = gh * gw
+        pos = None
+        if keep is not None:
+            k = int(n0 * keep)
+            pos_h = np.stack([np.sort(rng.choice(n0, size=k, replace=False)) for _ in range(B)]).astype(np.int32)
+            pos = torch.from_numpy(pos_h).to(ctx.device)
+            n0 = k
+        q, k_, v = synth.attention_qkv(300 + gh, B, G + n0, H, 64)
+        dq, dk, dv = (torch.from_numpy(a).to(ctx.device).to(torch.bfloat16) for a in (q, k_, v))
+        first, first_sc = None, None
+        for _ in range(5):
+            o, sc = ctx.spatial_block_attention(dq, dk, dv, gh, gw, b, r, n_global=G, patch_pos=pos, want_scores=True)
+            ctx.check()
+            if first is None:
+                first, first_sc = o.clone(), sc.clone()
+            else:
+                assert torch.equal(o.view(torch.int16), first.view(torch.int16))
+                assert torch.equal(sc.view(torch.int32), first_sc.view(torch.int32))
