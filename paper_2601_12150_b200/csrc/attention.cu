@@ -31,22 +31,18 @@ constexpr int TQ = 128;            // query rows per tile (MMA M)
 constexpr int TK = 32;             // keys per tile (MMA N of S, K extent of P V): three S buffers of 32 columns and
                                    // O make 160 TMEM columns, so three CTAs fit an SM
 constexpr int HD = 64;             // head_dim
-// K / V shared-memory stages (Q K^T runs up to two key tiles ahead of P V; an even count, so that each of the
-// two Q K^T issuers always meets the same stages): six with up to 8 global tokens, four with 9-16, whose rows and
-// scores take 10 KB more -- three CTAs fit an SM either way.
-constexpr int kst_for(int grows) { return grows <= 8 ? 6 : 4; }
+constexpr int KST = 6;             // K / V smem stages (Q K^T runs up to two key tiles ahead of P V; an even count, so
+                                   // that each of the two Q K^T issuers always meets the same stages)
 constexpr int NSB = 3;             // S / P buffers in TMEM: a softmax warp may be two key tiles ahead of the slowest
 constexpr int ATT_THREADS = 256;   // warps 0-3 softmax (one warpgroup), 4 TMA, 5-7 MMA issue: the second warpgroup
                                    // hands most of its registers to the first
 constexpr int TILE_BYTES = 128 * 128;  // Q tile
 constexpr int KV_BYTES = TK * 128;      // K or V tile
-constexpr int MAXG = 16;           // global tokens
-// Shared memory of a CTA for `grows` rows of global tokens (8 or 16):
-// Q tile, K / V stages, the global tokens' key and value rows (128 B each), barriers, their scores per query row.
-constexpr int att_smem(int grows) {
-  return TILE_BYTES + 2 * kst_for(grows) * KV_BYTES + 2 * grows * 128 + 1024 /*align*/ + 512 /*barriers*/ +
-         grows * 128 * 4;
-}
+constexpr int MAXG = 16;           // global tokens: they are the first key tile of every query tile (at most TK).
+                                   // (Adding them per query row in the epilogue with fp32 arithmetic instead was
+                                   // measured: equal at one global token, 5 / 17 / 28 % slower at 2 / 5 / 8.)
+// Shared memory of a CTA: Q tile, K / V stages, alignment slack, barriers.
+constexpr int ATT_SMEM = TILE_BYTES + 2 * KST * KV_BYTES + 1024 /*align*/ + 512 /*barriers*/;
 // two TMEM allocations per CTA, 160 columns in all, so that three CTAs share an SM's 512: O and two S buffers in
 // the first, the third S buffer in the second.  A row's P (bf16, 16 columns) is written over its own S.
 constexpr uint32_t TMEM_COLS = 128, TMEM_S2_COLS = 32;
@@ -251,7 +247,6 @@ struct PatchParams {
   __nv_bfloat16* o;
   int64_t o_sb, o_st, o_sh;
   int nbx, nby, nb, radius, n_global, n_patch, tiles_per_image;
-  int grows;                       // rows reserved for the global tokens in shared memory (8 or 16)
   float scale_log2;
   uint32_t* status;
 };
@@ -278,11 +273,9 @@ __device__ __forceinline__ void unpack8(const uint4& u, float* f) {
   }
 }
 
-template <int KST>
 __global__ void __launch_bounds__(ATT_THREADS, 3)
 attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kg,
-                  const __grid_constant__ CUtensorMap tm_vg, const __grid_constant__ CUtensorMap tm_o,
+                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                   const PatchParams p) {
   const int b = blockIdx.z, h = blockIdx.y;
   const int4 tile = __ldg(p.tiles + (size_t)b * p.tiles_per_image + blockIdx.x);
@@ -295,9 +288,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   uint8_t* sQ = smem;
   uint8_t* sK = smem + TILE_BYTES;
   uint8_t* sV = sK + KST * KV_BYTES;
-  uint8_t* sKg = sV + KST * KV_BYTES;      // global-token key rows (G x 128 B, swizzled)
-  uint8_t* sVg = sKg + p.grows * 128;                    // global-token value rows
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sVg + p.grows * 128);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + KST * KV_BYTES);
   uint64_t* q_full = bars;
   uint64_t* k_full = bars + 1;
   uint64_t* k_empty = k_full + KST;
@@ -308,7 +299,6 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   uint64_t* pv_done = p_full + NSB;      // [NSB] P V of the buffer's key tile (and all before it) has completed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + NSB);
   volatile uint32_t* abort_flag = tmem_slot + 3;
-  float* s_sg = reinterpret_cast<float*>(bars + 64);     // [G][128] scaled scores of the global keys
   static_assert(1 + 4 * KST + 3 * NSB + 2 <= 64, "barrier area");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -347,13 +337,14 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // ---------------- TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
-      mbar_expect_tx(q_full, TILE_BYTES + 2 * G * 128);
+      mbar_expect_tx(q_full, TILE_BYTES);
       tma_load_4d(sQ, &tm_q, q_full, 0, G + q_begin, h, b);
-      tma_load_4d(sKg, &tm_kg, q_full, 0, 0, h, b);
-      tma_load_4d(sVg, &tm_vg, q_full, 0, 0, h, b);
+      // The global tokens are the first key tile of every query tile: in the patch coordinates used here (key kb
+      // is token G + kb) they are the keys [-G, 0), a block row of their own in front of the neighbourhood's.
       uint32_t j = 0;
-      for (int cy = cy0; cy <= cy1; ++cy) {
-        const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
+      for (int cy = cy0 - 1; cy <= cy1; ++cy) {
+        int ks = -G, ke = 0;
+        if (cy >= cy0) { ks = __ldg(boff + cy * p.nbx + cxl); ke = __ldg(boff + cy * p.nbx + cxh + 1); }
         for (int kb = ks; kb < ke; kb += TK, ++j) {
           const int s = j % KST;
           const uint32_t ph = ((j / KST) & 1) ^ 1;
@@ -372,7 +363,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // consecutive tiles go to different S buffers) and O += P V one (warp 6; its instructions accumulate into the
     // same O and stay in one thread's order).
     if (lane == 0) {
-      uint32_t n_kv = 0;
+      uint32_t n_kv = 1;                                   // the global tokens' tile
       for (int cy = cy0; cy <= cy1; ++cy) {
         const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
         n_kv += (uint32_t)((ke - ks + TK - 1) / TK);
@@ -431,17 +422,18 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     // The running maximum starts at a finite floor instead of -inf, so that a tile in which this
     // row has no allowed key (all scores masked to -inf) gives p = 2^(-inf) = 0 and not 2^(nan).
-    // The global tokens join at the end (epilogue), while the last P V is still running.
+    // The first key tile holds the global tokens (allowed for every row), so l > 0 from then on.
     float m = -1.0e30f;
     float l = 0.f;
 
     uint32_t j = 0;
-    for (int cy = cy0; cy <= cy1; ++cy) {
-      const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
-      int lo = __ldg(boff + cy * p.nbx + rlo), hi = __ldg(boff + cy * p.nbx + rhi + 1);
-      // Rows past the end of the tile are never stored: they take the key range of the warp's
-      // first row, so that the warp stays uniform (valid rows are a prefix of the tile).
-      {
+    for (int cy = cy0 - 1; cy <= cy1; ++cy) {
+      int ks = -G, ke = 0, lo = -G, hi = 0;                // the global tokens' tile: keys [-G, 0) for every row
+      if (cy >= cy0) {
+        ks = __ldg(boff + cy * p.nbx + cxl); ke = __ldg(boff + cy * p.nbx + cxh + 1);
+        lo = __ldg(boff + cy * p.nbx + rlo); hi = __ldg(boff + cy * p.nbx + rhi + 1);
+        // Rows past the end of the tile are never stored: they take the key range of the warp's
+        // first row, so that the warp stays uniform (valid rows are a prefix of the tile).
         const int lo0 = __shfl_sync(0xffffffffu, lo, 0), hi0 = __shfl_sync(0xffffffffu, hi, 0);
         const bool v0 = __shfl_sync(0xffffffffu, (int)valid, 0) != 0;
         if (!valid) { lo = lo0; hi = v0 ? hi0 : lo0; }
@@ -533,75 +525,18 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_arrive(&p_full[sbuf]);
       }
     }
-    // ---------------- epilogue: the global tokens join the softmax, then O / l
-    // scaled scores of the global keys (their rows sit in shared memory since the Q tile arrived);
-    // computed before the wait for the last P V, which runs meanwhile
-    mbar_wait(q_full, 0, abort_flag, p.status, 0x1700);
-    float m_g = -INFINITY;
-    {
-      float qf[HD];
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const uint4 u = *reinterpret_cast<const uint4*>(sQ + row * 128 + ((c ^ (row & 7)) << 4));
-        unpack8(u, qf + 8 * c);
-      }
-#pragma unroll 1
-      for (int g = 0; g < G; ++g) {
-        float2 d[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {                              // eight independent chains, packed in pairs
-          float kf[8];
-          unpack8(*reinterpret_cast<const uint4*>(sKg + g * 128 + ((c ^ (g & 7)) << 4)), kf);
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            d[i] = __ffma2_rn(make_float2(qf[8 * c + 2 * i], qf[8 * c + 2 * i + 1]), make_float2(kf[2 * i], kf[2 * i + 1]), d[i]);
-        }
-        const float sc = (((d[0].x + d[0].y) + (d[1].x + d[1].y)) + ((d[2].x + d[2].y) + (d[3].x + d[3].y))) * sl2;
-        s_sg[g * 128 + row] = sc;
-        m_g = fmaxf(m_g, sc);
-      }
-    }
-    const float m_f = fmaxf(m, m_g);                 // finite: there is at least one global key
-    const float a_p = fast_exp2(m - m_f);            // weight of everything accumulated so far
-    float l_f = l * a_p;
-#pragma unroll 1
-    for (int g = 0; g < G; ++g) l_f += fast_exp2(s_sg[g * 128 + row] - m_f);
-    const float inv = 1.0f / l_f;
-    if (j > 0) {
-      mbar_wait(&pv_done[(j - 1) % NSB], ((j - 1) / NSB) & 1, abort_flag, p.status, 0x1A00);
-      tc_fence_after();
-    }
+    // ---------------- epilogue: O / l once the last P V has completed (l > 0: every row saw the global keys)
+    const float inv = 1.0f / l;
+    mbar_wait(&pv_done[(j - 1) % NSB], ((j - 1) / NSB) & 1, abort_flag, p.status, 0x1A00);
+    tc_fence_after();
     float of[HD];
-    {
-      const float a_o = a_p * inv;
 #pragma unroll
-      for (int c = 0; c < HD / 32; ++c) {
-        uint32_t orr[32];
-        if (j > 0) {
-          tmem_ld32(lane_addr + O_COL + 32 * c, orr);
-          tc_wait_ld();
-        } else {
+    for (int c = 0; c < HD / 32; ++c) {
+      uint32_t orr[32];
+      tmem_ld32(lane_addr + O_COL + 32 * c, orr);
+      tc_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) orr[i] = 0u;
-        }
-#pragma unroll
-        for (int i = 0; i < 32; ++i) of[32 * c + i] = __uint_as_float(orr[i]) * a_o;
-      }
-    }
-#pragma unroll 1
-    for (int g = 0; g < G; ++g) {
-      const float w = fast_exp2(s_sg[g * 128 + row] - m_f) * inv;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        float vf[8];
-        unpack8(*reinterpret_cast<const uint4*>(sVg + g * 128 + ((c ^ (g & 7)) << 4)), vf);
-#pragma unroll
-        for (int i = 0; i < 8; i += 2) {
-          const float2 t = __ffma2_rn(make_float2(w, w), make_float2(vf[i], vf[i + 1]), make_float2(of[8 * c + i], of[8 * c + i + 1]));
-          of[8 * c + i] = t.x;
-          of[8 * c + i + 1] = t.y;
-        }
-      }
+      for (int i = 0; i < 32; ++i) of[32 * c + i] = __uint_as_float(orr[i]) * inv;
     }
     // stage the bf16 row in the (now dead) Q tile, same 128-byte swizzle; each warp then stores its
     // own 32 rows, eight lanes per 128-byte row
@@ -943,17 +878,12 @@ int32_t spv_attn_plan_build(spv_ctx* ctx, int32_t batch, int32_t grid_h, int32_t
 
 int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, cudaStream_t stream) {
   if (!ctx->attn_configured) {
-    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel<kst_for(8)>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     att_smem(8)));
-    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel<kst_for(MAXG)>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     att_smem(MAXG)));
+    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM));
     ctx->attn_configured = 1;
   }
   const int n_tok = plan->n_global + plan->n_patch;
-  CUtensorMap tq, tk, tv, tkg, tvg;
+  CUtensorMap tq, tk, tv;
   int32_t st;
-  if ((st = make_qkv_map(ctx, &tkg, io->k, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, plan->n_global)) != SPV_OK) return st;
-  if ((st = make_qkv_map(ctx, &tvg, io->v, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, plan->n_global)) != SPV_OK) return st;
   if ((st = make_qkv_map(ctx, &tq, io->q, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TQ)) != SPV_OK) return st;
   if ((st = make_qkv_map(ctx, &tk, io->k, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TK)) != SPV_OK) return st;
   if ((st = make_qkv_map(ctx, &tv, io->v, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TK)) != SPV_OK) return st;
@@ -964,7 +894,6 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   pp.o = (__nv_bfloat16*)io->o; pp.o_sb = io->o_sb; pp.o_st = io->o_st; pp.o_sh = io->o_sh;
   pp.nbx = plan->nbx; pp.nby = plan->nby; pp.nb = plan->nb; pp.radius = plan->radius;
   pp.n_global = plan->n_global; pp.n_patch = plan->n_patch; pp.tiles_per_image = plan->tiles_per_image;
-  pp.grows = plan->n_global <= 8 ? 8 : MAXG;
   pp.scale_log2 = io->scale * 1.4426950408889634f;
   pp.status = ctx->d_status;
   const dim3 grid(plan->tiles_per_image, io->heads, plan->batch);
@@ -972,10 +901,7 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   // the output as a tensor map (same row order as Q, boxes of 32 rows): warps whose rows are all valid store by TMA
   CUtensorMap to;
   if ((st = make_qkv_map(ctx, &to, io->o, io->o_sb, io->o_st, io->o_sh, n_tok, io->heads, plan->batch, 32)) != SPV_OK) return st;
-  if (pp.grows == 8)
-    attn_patch_kernel<kst_for(8)><<<grid, ATT_THREADS, att_smem(8), stream>>>(tq, tk, tv, tkg, tvg, to, pp);
-  else
-    attn_patch_kernel<kst_for(MAXG)><<<grid, ATT_THREADS, att_smem(MAXG), stream>>>(tq, tk, tv, tkg, tvg, to, pp);
+  attn_patch_kernel<<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, to, pp);
   return spv_launch_ok(ctx);
 }
 
