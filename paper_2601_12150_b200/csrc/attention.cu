@@ -466,10 +466,13 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // c_lo <= c < c_hi, one unsigned compare
         if (!(kb >= ilo && kb + TK <= ihi)) {
           const int c_lo = min(max(lo - kb, 0), TK), c_hi = min(max(hi - kb, 0), TK);
-          const uint32_t width = (uint32_t)(c_hi - c_lo);
+          // bit i of the row's mask word = column i is allowed (bits [c_lo, c_hi))
+          const uint32_t below_hi = c_hi >= 32 ? 0xffffffffu : (1u << c_hi) - 1u;
+          const uint32_t below_lo = c_lo >= 32 ? 0xffffffffu : (1u << c_lo) - 1u;
+          const uint32_t mw = below_hi & ~below_lo;
 #pragma unroll
           for (int i = 0; i < TK; ++i)
-            if ((uint32_t)(i - c_lo) >= width) sr[i] = 0xff800000u;
+            if (!(mw & (1u << i))) sr[i] = 0xff800000u;
         }
         float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
