@@ -249,6 +249,13 @@ struct PatchParams {
   int nbx, nby, nb, radius, n_global, n_patch, tiles_per_image;
   float scale_log2;
   uint32_t* status;
+  // global-query form (template parameter GLOB): the query tile is the global tokens' rows, a CTA takes the key
+  // chunk blockIdx.x and leaves its (reference maximum, sum, sum p*v) per row for attn_global_combine
+  int chunk_len, n_chunks;
+  float scale;                     // natural-logarithm scale of the logits
+  float* logits;                   // [batch * G * heads, n_tok] scaled logits of global token 0's rows, or NULL
+  float* part_ml;                  // [batch * G * heads, n_chunks, 2]
+  float* part_o;                   // [batch * G * heads, n_chunks, 64]
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -273,15 +280,20 @@ __device__ __forceinline__ void unpack8(const uint4& u, float* f) {
   }
 }
 
+template <bool GLOB>
 __global__ void __launch_bounds__(ATT_THREADS, 3)
 attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                   const PatchParams p) {
   const int b = blockIdx.z, h = blockIdx.y;
-  const int4 tile = __ldg(p.tiles + (size_t)b * p.tiles_per_image + blockIdx.x);
+  // patch coordinates: key (and query) kb is token G + kb, so the global tokens are [-G, 0)
+  int4 tile = make_int4(-p.n_global, 0, 0, 0);           // global-query form: the query rows are the global tokens
+  if constexpr (!GLOB) tile = __ldg(p.tiles + (size_t)b * p.tiles_per_image + blockIdx.x);
   const int q_begin = tile.x, q_end = tile.y;
   if (q_begin >= q_end) return;                          // unused slot of the tile table
   const int by = tile.z, bx_first = tile.w & 0xFFFF, bx_last = tile.w >> 16;
+  // global-query form: this CTA's chunk of the keys (all of them are allowed)
+  const int gk0 = -p.n_global + (int)blockIdx.x * p.chunk_len, gk1 = min(gk0 + p.chunk_len, p.n_patch);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -303,7 +315,8 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = p.radius, G = p.n_global;
-  const int cy0 = max(by - r, 0), cy1 = min(by + r, p.nby - 1);
+  // the key ranges are walked block row by block row; the global-query form has one range, its chunk
+  const int cy0 = GLOB ? 1 : max(by - r, 0), cy1 = GLOB ? 0 : min(by + r, p.nby - 1);
   const int cxl = max(bx_first - r, 0), cxh = min(bx_last + r, p.nbx - 1);
   const int32_t* boff = p.block_off + (size_t)b * (p.nb + 1);
 
@@ -343,7 +356,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       // is token G + kb) they are the keys [-G, 0), a block row of their own in front of the neighbourhood's.
       uint32_t j = 0;
       for (int cy = cy0 - 1; cy <= cy1; ++cy) {
-        int ks = -G, ke = 0;
+        int ks = GLOB ? gk0 : -G, ke = GLOB ? gk1 : 0;
         if (cy >= cy0) { ks = __ldg(boff + cy * p.nbx + cxl); ke = __ldg(boff + cy * p.nbx + cxh + 1); }
         for (int kb = ks; kb < ke; kb += TK, ++j) {
           const int s = j % KST;
@@ -363,7 +376,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // consecutive tiles go to different S buffers) and O += P V one (warp 6; its instructions accumulate into the
     // same O and stay in one thread's order).
     if (lane == 0) {
-      uint32_t n_kv = 1;                                   // the global tokens' tile
+      uint32_t n_kv = GLOB ? (uint32_t)((gk1 - gk0 + TK - 1) / TK) : 1u;   // (patch form: the global tokens' tile)
       for (int cy = cy0; cy <= cy1; ++cy) {
         const int ks = __ldg(boff + cy * p.nbx + cxl), ke = __ldg(boff + cy * p.nbx + cxh + 1);
         n_kv += (uint32_t)((ke - ks + TK - 1) / TK);
@@ -416,7 +429,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
     const uint32_t lane_addr = tmem + lane_off;
     int bxq = bx_first;
-    if (valid) bxq = __ldg(p.tok_blk + (size_t)b * p.n_patch + tok) % p.nbx;
+    if (!GLOB && valid) bxq = __ldg(p.tok_blk + (size_t)b * p.n_patch + tok) % p.nbx;
     const int rlo = max(bxq - r, 0), rhi = min(bxq + r, p.nbx - 1);
     const float sl2 = p.scale_log2;
 
@@ -429,9 +442,12 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     uint32_t j = 0;
     for (int cy = cy0 - 1; cy <= cy1; ++cy) {
       int ks = -G, ke = 0, lo = -G, hi = 0;                // the global tokens' tile: keys [-G, 0) for every row
-      if (cy >= cy0) {
-        ks = __ldg(boff + cy * p.nbx + cxl); ke = __ldg(boff + cy * p.nbx + cxh + 1);
-        lo = __ldg(boff + cy * p.nbx + rlo); hi = __ldg(boff + cy * p.nbx + rhi + 1);
+      if constexpr (GLOB) { ks = lo = gk0; ke = hi = gk1; }
+      if (GLOB || cy >= cy0) {
+        if constexpr (!GLOB) {
+          ks = __ldg(boff + cy * p.nbx + cxl); ke = __ldg(boff + cy * p.nbx + cxh + 1);
+          lo = __ldg(boff + cy * p.nbx + rlo); hi = __ldg(boff + cy * p.nbx + rhi + 1);
+        }
         // Rows past the end of the tile are never stored: they take the key range of the warp's
         // first row, so that the warp stays uniform (valid rows are a prefix of the tile).
         const int lo0 = __shfl_sync(0xffffffffu, lo, 0), hi0 = __shfl_sync(0xffffffffu, hi, 0);
@@ -462,6 +478,15 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         uint32_t sr[TK];
         tmem_ld32(s_addr, sr);
         tc_wait_ld();
+        if constexpr (GLOB) {
+          // the scaled logits of global token 0 (query row 0) for the consumer of the CLS->patch scores
+          if (p.logits && row == 0) {
+            float* lg = p.logits + ((size_t)(b * G) * gridDim.y + h) * (size_t)(G + p.n_patch) + (G + kb);
+#pragma unroll
+            for (int i = 0; i < TK; ++i)
+              if (kb + i < ke) lg[i] = __uint_as_float(sr[i]) * p.scale;
+          }
+        }
         // a tile that is not inside every row's range is masked in registers: column c is allowed iff
         // c_lo <= c < c_hi, one unsigned compare
         if (!(kb >= ilo && kb + TK <= ihi)) {
@@ -532,6 +557,28 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const float inv = 1.0f / l;
     mbar_wait(&pv_done[(j - 1) % NSB], ((j - 1) / NSB) & 1, abort_flag, p.status, 0x1A00);
     tc_fence_after();
+    if constexpr (GLOB) {
+      // the chunk's partial state of the global rows, in the units attn_global_combine merges: reference maximum
+      // as a natural-logarithm logit (any reference does: sums and values are relative to it), sum, sum p * v
+      if (warp == 0) {                                     // the G <= 16 valid rows are rows of warp 0
+        const size_t pidx = ((size_t)(b * G + min(row, G - 1)) * gridDim.y + h) * p.n_chunks + blockIdx.x;
+        if (valid) {
+          p.part_ml[pidx * 2] = m * 0.6931471805599453f;
+          p.part_ml[pidx * 2 + 1] = l;
+        }
+#pragma unroll
+        for (int c = 0; c < HD / 32; ++c) {
+          uint32_t orr[32];
+          tmem_ld32(lane_addr + O_COL + 32 * c, orr);
+          tc_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              *reinterpret_cast<uint4*>(p.part_o + pidx * HD + 32 * c + i) = make_uint4(orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
+          }
+        }
+      }
+    } else {
     float of[HD];
 #pragma unroll
     for (int c = 0; c < HD / 32; ++c) {
@@ -582,6 +629,7 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if (q_begin + r0 + 4 * q4 < q_end) *reinterpret_cast<uint4*>(obase + (int64_t)ot[q4] * p.o_st) = w[q4];
       }
     }
+    }  // !GLOB
   }
   tc_fence_before();
   __syncthreads();
@@ -596,6 +644,8 @@ attn_patch_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 // global-query rows
 // ------------------------------------------------------------------------------------------
 constexpr int GCH = 128;   // fewest keys per CTA (bounds the number of chunk partials)
+constexpr int GLOB_TENSOR_MIN = 3;   // from this many global tokens on, their rows run as a query tile of the tensor-core
+                                     // kernel (measured equal at two, 1.6 to 5 times faster from three to sixteen)
 
 // grid (heads, chunks, batch * ceil(G / GQ)).  One pass over the chunk's keys serves GQ global queries (GQ = 1 is
 // what runs: with four queries per pass K and V cross HBM once per four queries, but the eight-lane dot products
@@ -879,14 +929,20 @@ int32_t spv_attn_plan_build(spv_ctx* ctx, int32_t batch, int32_t grid_h, int32_t
   return spv_launch_ok(ctx, launches);
 }
 
-int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, cudaStream_t stream) {
+static int32_t attn_configure(spv_ctx* ctx) {
   if (!ctx->attn_configured) {
-    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM));
+    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM));
+    SPV_CUDA_OK(cudaFuncSetAttribute(attn_patch_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM));
     ctx->attn_configured = 1;
   }
+  return SPV_OK;
+}
+
+int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAttnIO* io, cudaStream_t stream) {
+  int32_t st;
+  if ((st = attn_configure(ctx)) != SPV_OK) return st;
   const int n_tok = plan->n_global + plan->n_patch;
   CUtensorMap tq, tk, tv;
-  int32_t st;
   if ((st = make_qkv_map(ctx, &tq, io->q, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TQ)) != SPV_OK) return st;
   if ((st = make_qkv_map(ctx, &tk, io->k, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TK)) != SPV_OK) return st;
   if ((st = make_qkv_map(ctx, &tv, io->v, io->sb, io->st, io->sh, n_tok, io->heads, plan->batch, TK)) != SPV_OK) return st;
@@ -899,12 +955,13 @@ int32_t spv_attn_run_patches(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   pp.n_global = plan->n_global; pp.n_patch = plan->n_patch; pp.tiles_per_image = plan->tiles_per_image;
   pp.scale_log2 = io->scale * 1.4426950408889634f;
   pp.status = ctx->d_status;
+  pp.chunk_len = 0; pp.n_chunks = 0; pp.scale = io->scale; pp.logits = nullptr; pp.part_ml = nullptr; pp.part_o = nullptr;
   const dim3 grid(plan->tiles_per_image, io->heads, plan->batch);
   SpvProfScope prof(ctx, SPV_K_ATTN_PATCH, stream);
   // the output as a tensor map (same row order as Q, boxes of 32 rows): warps whose rows are all valid store by TMA
   CUtensorMap to;
   if ((st = make_qkv_map(ctx, &to, io->o, io->o_sb, io->o_st, io->o_sh, n_tok, io->heads, plan->batch, 32)) != SPV_OK) return st;
-  attn_patch_kernel<<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, to, pp);
+  attn_patch_kernel<false><<<grid, ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, to, pp);
   return spv_launch_ok(ctx);
 }
 
@@ -921,6 +978,44 @@ int32_t spv_attn_run_globals(spv_ctx* ctx, const SpvAttnPlan* plan, const SpvAtt
   const int n_tok = plan->n_global + plan->n_patch, G = plan->n_global, B = plan->batch;
   if (ws_bytes < spv_attn_global_bytes(B, G, io->heads, n_tok)) return SPV_ERR_WORKSPACE;
   const size_t rows = (size_t)B * G * io->heads;
+  if (G >= GLOB_TENSOR_MIN) {
+    // Several global tokens: their rows are one query tile of the tensor-core kernel (global-query form), the keys
+    // split into chunks so that the CTAs fill the GPU about once (three per SM); the chunk partials are merged by
+    // the same combine kernel.  One pass serves all G queries, so the time does not grow with G.
+    int32_t st;
+    if ((st = attn_configure(ctx)) != SPV_OK) return st;
+    int chunks = (int)(((size_t)ctx->sm_count * 3 + (size_t)B * io->heads - 1) / ((size_t)B * io->heads));
+    int chunk_len = ((n_tok + chunks - 1) / chunks + TK - 1) / TK * TK;
+    if (chunk_len < 2 * GCH) chunk_len = 2 * GCH;
+    chunks = (n_tok + chunk_len - 1) / chunk_len;
+    char* w = (char*)ws;
+    float* logits = (float*)w; w += spv_align_up(rows * n_tok * 4, 256);
+    float* part_ml = (float*)w; w += spv_align_up(rows * chunks * 2 * 4, 256);
+    float* part_o = (float*)w;
+    if (logits_out) *logits_out = logits;
+    CUtensorMap tq, tk, tv;
+    if ((st = make_qkv_map(ctx, &tq, io->q, io->sb, io->st, io->sh, n_tok, io->heads, B, TQ)) != SPV_OK) return st;
+    if ((st = make_qkv_map(ctx, &tk, io->k, io->sb, io->st, io->sh, n_tok, io->heads, B, TK)) != SPV_OK) return st;
+    if ((st = make_qkv_map(ctx, &tv, io->v, io->sb, io->st, io->sh, n_tok, io->heads, B, TK)) != SPV_OK) return st;
+    PatchParams pp;
+    pp.block_off = plan->block_off; pp.tok_blk = plan->tok_blk; pp.tiles = plan->tiles; pp.o_tok = nullptr;
+    pp.k = (const __nv_bfloat16*)io->k; pp.v = (const __nv_bfloat16*)io->v;
+    pp.sb = io->sb; pp.st = io->st; pp.sh = io->sh;
+    pp.o = (__nv_bfloat16*)io->o; pp.o_sb = io->o_sb; pp.o_st = io->o_st; pp.o_sh = io->o_sh;
+    pp.nbx = 1; pp.nby = 1; pp.nb = 0; pp.radius = 0;
+    pp.n_global = G; pp.n_patch = plan->n_patch; pp.tiles_per_image = 0;
+    pp.scale_log2 = io->scale * 1.4426950408889634f;
+    pp.status = ctx->d_status;
+    pp.chunk_len = chunk_len; pp.n_chunks = chunks; pp.scale = io->scale;
+    pp.logits = (scores || head_stats) ? logits : nullptr; pp.part_ml = part_ml; pp.part_o = part_o;
+    SpvProfScope prof(ctx, SPV_K_ATTN_GLOBAL, stream);
+    attn_patch_kernel<true><<<dim3(chunks, io->heads, B), ATT_THREADS, ATT_SMEM, stream>>>(tq, tk, tv, tq, pp);
+    attn_global_combine<<<dim3(io->heads, B * G), 256, 0, stream>>>(logits, part_ml, part_o, chunks, n_tok, G,
+                                                                   io->heads, (__nv_bfloat16*)io->o, io->o_sb,
+                                                                   io->o_st, io->o_sh, scores, score_idx, score_stride,
+                                                                   head_stats);
+    return spv_launch_ok(ctx, 2);
+  }
   // as many chunks as fill the GPU once (two CTAs of this kernel per SM), none shorter than GCH keys
   const int max_chunks = (n_tok + GCH - 1) / GCH;
   const size_t ctas_per_chunk = (size_t)B * G * io->heads;

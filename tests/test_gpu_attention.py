@@ -108,7 +108,8 @@ def test_single_attention_op_28x28(ctx):
     (20, 20, 16, 0, 1, 1, 2),     # blocks larger than a tile (256 tokens), own block only
     (9, 30, 4, 3, 1, 2, 1),       # wide neighbourhood
     (12, 12, 1, 1, 1, 1, 2),      # one patch per block: 3x3-patch windows, a query tile per grid row
-    (10, 14, 3, 0, 8, 1, 1),      # own block only, eight global tokens (the most that leave three CTAs per SM)
+    (10, 14, 3, 0, 8, 1, 1),      # own block only, eight global tokens
+    (64, 64, 8, 1, 5, 1, 2),      # five global tokens over 4096 patches: their rows span several key chunks
     (18, 11, 8, 1, 9, 1, 2),      # nine global tokens (CLS + eight registers)
     (16, 24, 8, 1, 16, 2, 1),     # the maximum of sixteen global tokens
     (5, 3, 8, 1, 1, 1, 1),        # a grid smaller than one block
