@@ -954,11 +954,33 @@ def run_sweep(args):
             torch.cuda.synchronize()
             ctx.check()
             ms = e0.elapsed_time(e1) / steps
+            # small images are bound by the ~240 launches of a forward: the same call captured once in a
+            # CUDA graph and replayed (vit_forward only enqueues work on its stream)
+            ms_graph = None
+            if side <= args.sweep_graph_max_side:
+                out, _ = ctx.vit_forward(cfg, dw, img, g, g)
+                st = torch.cuda.Stream()
+                st.wait_stream(torch.cuda.current_stream())
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(st):
+                    with torch.cuda.graph(graph, stream=st):
+                        ctx.vit_forward(cfg, dw, img, g, g, out=out, stream=st)
+                graph.replay()
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(steps):
+                    graph.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                ctx.check()
+                ms_graph = e0.elapsed_time(e1) / steps
+                del graph
             fl = forward_flops(dict(wl, cfg=dict(cfg, radius=g if mode == "dense" else 1)),
                                None if kept is None else kept.cpu().numpy())
             useful = fl["gemm"] + fl["attn_patch"] + fl["attn_global"]
             print(json.dumps({"workload": wl["name"], "image": f"{side}x{side}", "tokens": 1 + g * g, "mode": mode,
                               "batch": B, "ms_per_step": ms, "images_per_s": B / (ms * 1e-3),
+                              "ms_per_step_graph_replay": ms_graph,
                               "useful_tflops": useful / (ms * 1e-3) / 1e12,
                               "frac_of_bf16_peak": useful / (ms * 1e-3) / 1e12 / pk["tensor"],
                               "attention_density": fl["attn_patch"] / max(1.0, forward_flops(
@@ -985,6 +1007,8 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="resolution sweep (dense / sparse / sparse+filter), one JSON line per point")
     ap.add_argument("--sweep-sides", default="224,448,1024,2048,3072,4096")
+    ap.add_argument("--sweep-graph-max-side", type=int, default=2048,
+                    help="largest image side of the sweep that is also timed as a CUDA-graph replay")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
