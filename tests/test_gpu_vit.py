@@ -200,7 +200,7 @@ def test_vit_forward_one_stage_list_equals_single_fields(ctx):
     assert np.array_equal(a, b) and np.array_equal(ka, kb)
 
 
-@pytest.mark.parametrize("stages,G", [([(1, 0.5)], 1), ([(1, 0.7), (2, 0.45)], 2)])
+@pytest.mark.parametrize("stages,G", [([(1, 0.5)], 1), ([(1, 0.7), (2, 0.45)], 2), ([(1, 0.6)], 5)])
 def test_fused_filter_front_end_is_bit_identical(ctx, stages, G):
     """The filter's fused front end (softmax weights of the CLS row, head mean and ranking keys in one kernel,
     no [batch, heads, patches] score tensor) keeps exactly the tokens the two separate kernels keep."""
